@@ -80,6 +80,7 @@ int svdmlp_forward(svdmlp_t* h, const void* X, int T, void* Y, void* stream);
  * returning.  For full copy overlap the host buffers should be page-locked.  On a non-default stream the
  * three operations of a call are recorded as one graph, which later calls with the same X_host, Y_host
  * and T replay (one launch instead of three); the buffers' contents may of course change between calls.
+ * The first call allocates the device-side staging copies of X and Y ([max_T, d] each).
  */
 int svdmlp_forward_host(svdmlp_t* h, const void* X_host, int T, void* Y_host, void* stream);
 
@@ -88,6 +89,9 @@ int svdmlp_forward_host(svdmlp_t* h, const void* X_host, int T, void* Y_host, vo
  *   h_out = h_in + MLP(RMSNorm(h_in)),  RMSNorm(h)[t, :] = h[t, :] / sqrt(mean(h[t, :]^2) + eps)
  * with unit norm weight.  h_in, h_out are fp32 [T, d] (the residual stream stays fp32; the
  * normalised rows are rounded to bf16 as the MLP input).  h_out may alias h_in.
+ * For T <= 8 normalisation and residual add run inside the decode kernel.  Otherwise the normalised
+ * rows pass through a [max_T, d] bf16 buffer that the first such call allocates (cudaMalloc may
+ * synchronise the device, so make that call before any stream capture).
  */
 int svdmlp_forward_prenorm_residual(svdmlp_t* h, const float* h_in, float* h_out, int T,
                                     float eps, void* stream);
@@ -114,8 +118,9 @@ size_t svdlinear_workspace_bytes(int T, int in, int out, int r);
  * loads the library holds SVDLINEAR_NOALLOC_MAX_ELEMS * 4 bytes (128 KiB) for it until exit.
  *
  * Same arguments and result as svdlinear_forward minus the workspace.  Limits: T <=
- * SVDLINEAR_NOALLOC_MAX_T and T * r <= SVDLINEAR_NOALLOC_MAX_ELEMS, otherwise
- * SVDMLP_ERR_UNSUPPORTED is returned and nothing is launched.  The call performs no cudaMalloc,
+ * SVDLINEAR_NOALLOC_MAX_T, T * r <= SVDLINEAR_NOALLOC_MAX_ELEMS and r <= SVDLINEAR_NOALLOC_MAX_R
+ * (the second kernel holds an 8-token strip of Z in shared memory, 32 (r + 32) bytes of the 227 KiB
+ * an SM has), otherwise SVDMLP_ERR_UNSUPPORTED is returned and nothing is launched.  The call performs no cudaMalloc,
  * cudaFree or other allocating call.  The first call on each device looks up the device address
  * of the array (one cudaGetSymbolAddress with that device current); make that first call before
  * any stream capture begins.  All calls on a device share the one array: it keeps the previous
@@ -125,6 +130,7 @@ size_t svdlinear_workspace_bytes(int T, int in, int out, int r);
  */
 #define SVDLINEAR_NOALLOC_MAX_T 32
 #define SVDLINEAR_NOALLOC_MAX_ELEMS 32768
+#define SVDLINEAR_NOALLOC_MAX_R 7232
 int svdlinear_forward_noalloc(const void* X, int T, int in, int out, int r, const void* U,
                               const void* V, void* Y, void* stream);
 
@@ -149,43 +155,6 @@ const char* svdmlp_strerror(int status);
  * gives up (SVDMLP_OK if none did).  The word is cleared by the call.
  */
 int svdmlp_last_device_status(svdmlp_t* h);
-
-/*
- * Failure-detection self-test.  Enqueues a one-warp kernel that waits - through the same bounded-wait routine
- * every production kernel uses - on a barrier that nothing will ever signal, with a limit of `limit_us`
- * microseconds (1 .. 1000000) instead of the production limit of 2 s.  When the limit passes the kernel
- * records SVDMLP_ERR_TIMEOUT in the handle's device status word and returns normally: nothing faults or traps,
- * the context and the handle stay usable, and svdmlp_last_device_status reports (and clears) the timeout.
- * Setting SVDMLP_LOG=1 in the environment makes forward calls print the kernel path they choose (stderr).
- */
-int svdmlp_selftest_timeout(svdmlp_t* h, unsigned limit_us, void* stream);
-
-/* Number of kernels this handle has launched since creation (for benchmark accounting). */
-unsigned long long svdmlp_launch_count(const svdmlp_t* h);
-
-/*
- * Per-kernel timing for benchmarks.  With profiling enabled every later forward call records a
- * CUDA event pair around each kernel it launches on the call's stream (a small serialising
- * overhead; leave it off for throughput runs and stream capture).  svdmlp_profile_read waits
- * for the most recent forward, writes the duration in milliseconds of each of its kernels to
- * ms[0 .. min(count, capacity)) in launch order and returns count (or a negative status);
- * svdmlp_profile_name gives the kernel's label ("stage1", "gateup", ...), NULL if out of range.
- */
-int svdmlp_profile_enable(svdmlp_t* h, int enable);
-int svdmlp_profile_read(svdmlp_t* h, float* ms, int capacity);
-const char* svdmlp_profile_name(const svdmlp_t* h, int index);
-
-/*
- * Measurement aid: restrict later forward calls of this handle to a subset of the path's kernels
- * so that one kernel can be timed or profiled back to back.  Bits: 1 first projection
- * (X V^T), 2 gate/up expansion with SiLU (small T: fused with the first half of the down chain),
- * 4 first half of the down chain (large T only), 8 second half of the down chain, 16 RMSNorm.
- * With anything but all bits set the outputs are meaningless.  Default: all bits.
- */
-int svdmlp_stage_mask(svdmlp_t* h, unsigned mask);
-
-/* Name of the kernel path the handle would use for T tokens: "skinny" or "tensor". */
-const char* svdmlp_path_name(const svdmlp_t* h, int T);
 
 #ifdef __cplusplus
 }

@@ -195,11 +195,12 @@ def svdlinear_forward(X, U, V, Y=None, workspace=None, stream=None) -> torch.Ten
 
 NOALLOC_MAX_T = 32
 NOALLOC_MAX_ELEMS = 32768
+NOALLOC_MAX_R = 7232
 
 
 def svdlinear_forward_noalloc(X, U, V, Y, stream=None) -> torch.Tensor:
     """XUV operator for callers that must not allocate: Y is caller-provided and the library's
-    built-in 128 KiB scratch array holds the intermediate (T <= 32, T * r <= 32768).  Calls that
+    built-in 128 KiB scratch array holds the intermediate (T <= 32, T * r <= 32768, r <= 7232).  Calls that
     may overlap on the GPU race on that array; the first call per device should precede any
     stream capture."""
     T, n_in = X.shape

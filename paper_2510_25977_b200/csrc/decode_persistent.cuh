@@ -278,29 +278,6 @@ __device__ __forceinline__ void red_add_v2(float* addr, float a, float b) {
     asm volatile("red.relaxed.gpu.global.add.v2.f32 [%0], {%1, %2};" ::"l"(addr), "f"(a), "f"(b) : "memory");
 }
 
-// Optional tuning aid (compile with -DSVDMLP_TIMELINE): thread 0 of every CTA records %globaltimer at
-// phase boundaries; svdmlp_timeline_read copies the table to the host.
-#ifdef SVDMLP_TIMELINE
-__device__ unsigned long long g_timeline[160 * 16];
-__device__ unsigned long long g_dbg[160 * 32];
-#define SVDMLP_TL(i) do { if (threadIdx.x == 0) g_timeline[blockIdx.x * 16 + (i)] = (unsigned long long)clock64(); } while (0)
-__device__ __forceinline__ void probe_load(int slot, const float* addr) {
-    if (threadIdx.x != 0) return;
-    long long c0, c1;
-    asm volatile("mov.u64 %0, %%clock64;" : "=l"(c0) :: "memory");
-    float y;
-    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(y) : "l"(addr) : "memory");
-    asm volatile("add.f32 %0, %0, 0f3F800000;" : "+f"(y) :: "memory");
-    asm volatile("mov.u64 %0, %%clock64;" : "=l"(c1) :: "memory");
-    if (y == 123.f) c1 += 1;
-    g_timeline[blockIdx.x * 16 + slot] = g_timeline[blockIdx.x * 16 + 0] + (unsigned long long)(c1 - c0);
-}
-#define SVDMLP_PROBE(i, a) probe_load(i, a)
-#else
-#define SVDMLP_TL(i) do {} while (0)
-#define SVDMLP_PROBE(i, a) do {} while (0)
-#endif
-
 struct Params {
     Shape s;
     CUtensorMap mX;                               // x_tma: X as [64 columns][T rows][d/64 column blocks], box [64][T][ga/4]
@@ -454,7 +431,6 @@ mlp_kernel(const __grid_constant__ Params p) {
     }
 
     // ---------------- consumers ----------------
-    SVDMLP_TL(0);
     Cursor cur;
     bool dead = false;  // a wait gave up: keep walking (every named barrier is still reached) without waiting
     int nwaited = 0;  // diagnostics: index of the group a consumer wait gave up on
@@ -543,7 +519,6 @@ mlp_kernel(const __grid_constant__ Params p) {
                     consumer_bar();
                 }
                 wait();
-                if (q == 0) SVDMLP_TL(12);
                 const unsigned char* vs = ring.slot(cur) + L.a_v_off;
                 const unsigned char* xs = fused_norm ? xn : p.x_res ? xres : ring.slot(cur);
                 const bool swz = p.x_tma && !fused_norm;
@@ -604,7 +579,6 @@ mlp_kernel(const __grid_constant__ Params p) {
                 release();
                 if (fused_norm && q + 1 < nga) consumer_bar();  // xn is rewritten for the next group
             }
-            SVDMLP_TL(13);
             float* red = reinterpret_cast<float*>(rest + L.red);  // [warp][16 MT tokens][8 NTA rows]
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt)
@@ -626,13 +600,11 @@ mlp_kernel(const __grid_constant__ Params p) {
             }
         }
     }
-    SVDMLP_TL(1);
     // A -> B hand-over.  The arrival count is only a hint that Z is probably complete (no fence orders the Z
     // stores before it); what makes the hand-over safe is that Z carries its own validity: an element that
     // has not been stored yet still holds kZUnset (phase D resets it), and the staging loop below re-reads
     // until none is left.  This saves the fence's round trip through a loaded memory system.
     if (!grid_arrive_wait<false>(p.bar + 2 * kBarStride, target, ring.abort)) dead = true;
-    SVDMLP_TL(2);
 
     unsigned char* zs = rest + L.zs;
     if (pb.count > 0) {
@@ -682,14 +654,12 @@ mlp_kernel(const __grid_constant__ Params p) {
                             *reinterpret_cast<uint4*>(zs + (tb + nrg * a) * L.pitch_z + pos * 2) = v[a][c];
                         }
             }
-        SVDMLP_TL(9);
         if (r16 != r)
             for (int idx = tid; idx < s.T * 2 * (r16 - r); idx += kConsumers) {
                 const int t = idx / (2 * (r16 - r)), rem = idx - t * 2 * (r16 - r), hf = rem / (r16 - r), k = r + rem - hf * (r16 - r);
                 *reinterpret_cast<__half*>(zs + t * L.pitch_z + (hf * r16 + k) * 2) = __float2half_rn(0.f);
             }
         consumer_bar();
-        SVDMLP_TL(3);
 
         // gate/up expansion: warp task = (tile, gate | up) over the full K = r
         const int ntask = 2 * pb.count, kg = s.kg_b(pb.count);
@@ -701,7 +671,6 @@ mlp_kernel(const __grid_constant__ Params p) {
         for (int k0 = 0; k0 < ksr; k0 += kg) {
             const int ns = min(kg, ksr - k0);
             wait();
-            if (k0 == 0) SVDMLP_TL(10);
             const unsigned char* slot = ring.slot(cur);
 #pragma unroll
             for (int it = 0; it < 2; ++it) {
@@ -722,7 +691,6 @@ mlp_kernel(const __grid_constant__ Params p) {
             }
             release();
         }
-        SVDMLP_TL(7);
         // SiLU(gate) .* up through shared memory: gate tasks publish G, up tasks build H (fp16)
         float* gs = reinterpret_cast<float*>(rest + L.gs);
         unsigned char* hs = rest + L.hs;
@@ -752,16 +720,13 @@ mlp_kernel(const __grid_constant__ Params p) {
             }
         }
         consumer_bar();
-        SVDMLP_TL(8);
 
         // first half of the down chain: Zd[:, 16-row tile] += H[:, cols of this CTA] Vd[tile, cols]^T
         const int gz = s.gz_b(pb.count);
         float* zdc = zd_cur + (size_t)(b % kCopiesZd) * zd_elems;
         for (int z0 = 0; z0 < zt; z0 += gz) {
             const int nz = min(gz, zt - z0);
-            if (z0 == 0) SVDMLP_TL(14);
             wait();
-            if (z0 == 0) SVDMLP_TL(11);
             const unsigned char* slot = ring.slot(cur);
             for (int z = warp; z < nz; z += kNW) {
                 float a2[NT][4];
@@ -798,9 +763,7 @@ mlp_kernel(const __grid_constant__ Params p) {
             release();
         }
     }
-    SVDMLP_TL(4);
     if (!grid_arrive_wait<true>(p.bar, target, ring.abort)) dead = true;
-    SVDMLP_TL(5);
     // every CTA staged Z before it arrived at the barrier: mark this CTA's entries unset for the next launch
     for (int idx = tid; idx < s.T * pa.count; idx += kConsumers) {
         const int t = idx / pa.count, c = idx - t * pa.count;
@@ -888,7 +851,6 @@ mlp_kernel(const __grid_constant__ Params p) {
             }
         }
     }
-    SVDMLP_TL(6);
     // every CTA has read the launch number before it arrived at the second barrier: bump it for the next launch
     if (b == 0 && tid == 0) p.bar[kBarStride] = epoch + 1ull;
     if (*ring.abort && p.status != nullptr && lane == 0) atomicExch(p.status, -7);

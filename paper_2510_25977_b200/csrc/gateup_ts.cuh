@@ -167,10 +167,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_ts_pair_kernel(const _
             int stage = 0, cur_mp = -1, n = 0, mp = 0;
             uint32_t phase = 0, ph = 0, strip_phase = 0;
             bool ok = true;
-#ifdef SVDMLP_TIMELINE
-            const bool tl_on = blockIdx.x == 0 && threadIdx.x == 32;
-            int tl_n = 0;
-#endif
             auto skip_slots = [&](int k) { stage += k; while (stage >= nslot) { stage -= nslot; phase ^= 1; } };
             if (tile_begin < tile_end) { mp = tile_begin / p.tiles_n; n = tile_begin - mp * p.tiles_n; }
             for (int t = tile_begin; t < tile_end && ok; ++t) {
@@ -209,16 +205,12 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_ts_pair_kernel(const _
                 }
                 if (b == 1) skip_slots(spb);  // G's slots of this tile
                 // this branch's accumulator columns have been read out by every epilogue warp of both CTAs
-                GEMM_TL(1);
                 ok = umma::mbar_wait_warp(&tempty[b], ph ^ 1, abort_flag);
                 if (!ok) break;
-                GEMM_TL(2);
                 umma::tc_fence_after_sync();
                 for (int c = 0; c < chunks; c += 2) {
-                    GEMM_TL(4);
                     ok = umma::mbar_wait_warp(&full[stage], phase, abort_flag);
                     if (!ok) break;
-                    GEMM_TL(5);
                     if (umma::elect_one()) {
                         const uint64_t bd0 = umma::smem_desc_sw128(umma::smem_u32(ring + stage * kTsSlotBytes));
                         const uint32_t dcol = tmem_base + 256 + b * 128, acol = tmem_base + b * 128 + c * 32;
@@ -244,9 +236,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_ts_pair_kernel(const _
                 if (b == 0) skip_slots(spb);  // Up's slots of this tile
                 if (++n == p.tiles_n) { n = 0; ++mp; }
             }
-#ifdef SVDMLP_TIMELINE
-            if (tl_on) { g_gemm_tl[0] = tl_n; g_gemm_tl[1] = tile_end - tile_begin; }
-#endif
         }
     } else if (warp < 2 + kEpiWarps) {  // ---------------- epilogue warps 2..9 (both CTAs, own 128 rows) ----------------
         const int q = warp & 3, half = (warp - 2) >> 2;
@@ -255,19 +244,13 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_ts_pair_kernel(const _
         const uint32_t tempty_g = umma::map_to_rank(&tempty[0], 0), tempty_u = umma::map_to_rank(&tempty[1], 0);
         unsigned char* my_stage = stage_out + (warp - 2) * 4096;
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + 256 + half * 64;
-#ifdef SVDMLP_TIMELINE
-        const bool tl_on = blockIdx.x == 0 && threadIdx.x == 64;
-        int tl_n = 1020;
-#endif
         int mp = tile_begin / p.tiles_n, n = tile_begin - mp * p.tiles_n;
         for (int t = tile_begin; t < tile_end && ok; ++t, (++n == p.tiles_n ? (n = 0, ++mp) : 0)) {
             const int m = 2 * mp + (int)rank;
             uint32_t rr[2][32], sg[32];
             // G: this warp's 32 rows x 64 columns into registers, then its columns go back to the issuer
-            GEMM_TL(11);
             ok = umma::mbar_wait_warp(&tfull[0], ph, abort_flag);
             if (!ok) break;
-            GEMM_TL(12);
             umma::tc_fence_after_sync();
             umma::tmem_ld32(taddr, rr[0]);
             umma::tmem_ld32(taddr + 32, rr[1]);
@@ -275,7 +258,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_ts_pair_kernel(const _
             umma::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) umma::mbar_arrive_cluster(tempty_g);
-            GEMM_TL(13);
             // SiLU(G) = h + h tanh(h), h = G / 2, as packed fp16 while the tensor pipe is still busy with Up: the
             // MUFU-bound part of the epilogue (1024 cycles per tile and scheduler) hides behind Up's MMAs.
 #pragma unroll
@@ -288,11 +270,9 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_ts_pair_kernel(const _
                     const __half2 s2 = __hfma2(h2, *reinterpret_cast<const __half2*>(&t2), h2);
                     sg[hh * 16 + j] = *reinterpret_cast<const uint32_t*>(&s2);
                 }
-            GEMM_TL(16);
             // Up likewise, multiplied in as it arrives
             ok = umma::mbar_wait_warp(&tfull[1], ph, abort_flag);
             if (!ok) break;
-            GEMM_TL(14);
             umma::tc_fence_after_sync();
             umma::tmem_ld32(taddr + 128, rr[0]);
             umma::tmem_ld32(taddr + 160, rr[1]);
@@ -300,7 +280,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_ts_pair_kernel(const _
             umma::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) umma::mbar_arrive_cluster(tempty_u);
-            GEMM_TL(15);
             ph ^= 1;
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh)
@@ -323,11 +302,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_ts_pair_kernel(const _
                 umma::tma_store_2d(&p.tmC, my_stage, col, m * BM + q * 32);
                 umma::bulk_commit();
             }
-            GEMM_TL(17);
         }
-#ifdef SVDMLP_TIMELINE
-        if (tl_on) g_gemm_tl[4095] = tl_n;
-#endif
         umma::bulk_wait_all();
     }
 

@@ -3,6 +3,7 @@
 // streaming) and tensor_gemm.cuh (large T, tcgen05); this file only validates arguments,
 // owns the workspace, encodes TMA tensor maps and enqueues launches.
 #include "../../include/svdmlp.h"
+#include "../../include/svdmlp_bench.h"
 
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -947,13 +948,13 @@ int svdmlp_forward_prenorm_residual(svdmlp_t* h, const float* h_in, float* h_out
         return SVDMLP_ERR_INVALID_ARG;
     if (!aligned16(h_in) || !aligned16(h_out)) return SVDMLP_ERR_ALIGNMENT;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (h->Xn == nullptr) {
-        if (cudaMalloc((void**)&h->Xn, (size_t)h->max_T * h->d * 2) != cudaSuccess) { cudaGetLastError(); return SVDMLP_ERR_NOMEM; }
-    }
     h->prof_n = 0;
     if (T <= 8 && use_skinny(h, T) && h->stage_mask == ~0u) {  // small T: RMSNorm inside the persistent decode kernel
         const int rc = skinny_forward(h, nullptr, T, h_out, 1, h_in, s, h_in, eps);
         if (rc != SVDMLP_ERR_UNSUPPORTED) return rc;
+    }
+    if (h->Xn == nullptr) {  // first call that needs the normalised rows in global memory
+        if (cudaMalloc((void**)&h->Xn, (size_t)h->max_T * h->d * 2) != cudaSuccess) { cudaGetLastError(); return SVDMLP_ERR_NOMEM; }
     }
     if (h->stage_mask & 16u) {
         ProfScope ps(h, "rmsnorm", s);
@@ -1004,7 +1005,18 @@ int svdmlp_selftest_timeout(svdmlp_t* h, unsigned limit_us, void* stream) {
 
 int svdmlp_stage_mask(svdmlp_t* h, unsigned mask) {
     if (h == nullptr) return SVDMLP_ERR_INVALID_ARG;
+    const bool restore = mask == ~0u && h->stage_mask != ~0u;
     h->stage_mask = mask;
+    if (restore) {
+        // a partial mask breaks the chain in which neighbouring kernels clear each other's accumulators:
+        // put the workspace back into the state a full forward expects
+        CUDA_TRY(cudaDeviceSynchronize());
+        if (h->Zs) CUDA_TRY(cudaMemset(h->Zs, 0, (size_t)h->t_skinny * (h->rg + h->ru) * 4));
+        if (h->Zds) CUDA_TRY(cudaMemset(h->Zds, 0, (size_t)h->t_skinny * h->rd * 4));
+        const int rr = persist_reset(h, nullptr);
+        if (rr != SVDMLP_OK) return rr;
+        CUDA_TRY(cudaDeviceSynchronize());
+    }
     return SVDMLP_OK;
 }
 
@@ -1074,15 +1086,19 @@ extern "C" int svdlinear_forward_noalloc(const void* X, int T, int in, int out, 
     if (!X || !U || !V || !Y || T <= 0 || in <= 0 || out <= 0 || r <= 0) return SVDMLP_ERR_INVALID_ARG;
     if ((in | out | r) & 7) return SVDMLP_ERR_ALIGNMENT;
     if (!aligned16(X) || !aligned16(U) || !aligned16(V) || !aligned16(Y)) return SVDMLP_ERR_ALIGNMENT;
-    if (T > SVDLINEAR_NOALLOC_MAX_T || (long)T * r > SVDLINEAR_NOALLOC_MAX_ELEMS) return SVDMLP_ERR_UNSUPPORTED;
+    if (T > SVDLINEAR_NOALLOC_MAX_T || (long)T * r > SVDLINEAR_NOALLOC_MAX_ELEMS || r > SVDLINEAR_NOALLOC_MAX_R)
+        return SVDMLP_ERR_UNSUPPORTED;
+    using namespace skinny;
+    // the second kernel keeps a [8 nt, r] strip of Z (as a hi + lo bf16 pair) in shared memory: settle the token
+    // tile and check that it fits before anything is enqueued
+    int nt = T <= 8 ? 1 : T <= 16 ? 2 : 4;
+    while (nt > 1 && (size_t)nt * 8 * 2 * (r + kPad) * 2 > 227 * 1024) nt >>= 1;
+    if ((size_t)nt * 8 * 2 * (r + kPad) * 2 > 227 * 1024) return SVDMLP_ERR_UNSUPPORTED;
     int rc = check_arch();
     if (rc != SVDMLP_OK) return rc;
     float* z = nullptr;
     if ((rc = noalloc_scratch(&z)) != SVDMLP_OK) return rc;
-    using namespace skinny;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int nt = T <= 8 ? 1 : T <= 16 ? 2 : 4;
-    while (nt > 1 && (size_t)nt * 8 * 2 * (r + kPad) * 2 > 227 * 1024) nt >>= 1;
     const int kc = 256;
     const int chunks = (T + nt * 8 - 1) / (nt * 8);
     dim3 g1(((r + 15) / 16 + 3) / 4, (in + kc - 1) / kc, chunks), g2((out + 63) / 64, 1, chunks);
@@ -1192,17 +1208,3 @@ int svdlinear_forward(const void* X, int T, int in, int out, int r, const void* 
 
 }  // extern "C"
 
-#ifdef SVDMLP_TIMELINE
-// Tuning aid, only in builds with -DSVDMLP_TIMELINE: copies the persistent decode kernel's per-CTA
-// phase timestamps (160 x 16 values, nanoseconds of %globaltimer) to `out`.
-extern "C" int svdmlp_timeline_read(unsigned long long* out) {
-    return cudaMemcpyFromSymbol(out, dpersist::g_timeline, sizeof(unsigned long long) * 160 * 16) == cudaSuccess ? 0 : -4;
-}
-extern "C" int svdmlp_gemm_timeline_read(long long* out) {
-    return cudaMemcpyFromSymbol(out, tensorpath::g_gemm_tl, sizeof(long long) * 4096) == cudaSuccess ? 0 : -4;
-}
-extern "C" int svdmlp_dbg_read(unsigned long long* out) {
-    return cudaMemcpyFromSymbol(out, dpersist::g_dbg, sizeof(unsigned long long) * 160 * 32) == cudaSuccess ? 0 : -4;
-}
-
-#endif

@@ -488,13 +488,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 // Barriers: loads of both CTAs complete on the leader's (rank 0) "full"/"afull" barriers; the
 // leader's MMA commits are multicast to the "empty"/"tfull"/"aempty" barriers of both CTAs; the
 // epilogue warps of both CTAs arrive on the leader's "tempty".
-#ifdef SVDMLP_TIMELINE
-// Tuning aid: (kind, clock) pairs recorded by the MMA issuer of cluster 0.
-__device__ long long g_gemm_tl[4096];
-#define GEMM_TL(kind) do { if (tl_on && tl_n < 2040) { g_gemm_tl[2 + tl_n] = ((long long)(kind) << 56) | (clock64() & 0xFFFFFFFFFFFFFFll); ++tl_n; } } while (0)
-#else
-#define GEMM_TL(kind) do { } while (0)
-#endif
 template <int NB, int BN, bool ARES>
 __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid_constant__ GemmParams p) {
     constexpr int HB_BYTES = (BN / 2) * BK * 2;  // this CTA's half of one B chunk
@@ -641,46 +634,27 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
             int stage = 0, cur_mp = -1, acc = 0;
             uint32_t phase = 0, a_phase = 0, acc_phase0 = 0, acc_phase1 = 0;
             bool ok = true;
-#ifdef SVDMLP_TIMELINE
-            #if defined(GEMM_TL_DOWN1)
-            const bool tl_on = !ARES && NB == 1 && p.ksplit > 1 && p.K > 4096 && blockIdx.x == 0 && threadIdx.x == 32;
-#elif defined(GEMM_TL_DOWN2)
-            const bool tl_on = NB == 1 && p.resid != nullptr && blockIdx.x == 0 && threadIdx.x == 32;
-#elif defined(GEMM_TL_TS)
-            const bool tl_on = false;
-#elif defined(GEMM_TL_WIDE)
-            const bool tl_on = !ARES && NB == 2 && blockIdx.x == 0 && threadIdx.x == 32;
-#else
-            const bool tl_on = ARES && NB == 2 && blockIdx.x == 0 && threadIdx.x == 32;
-#endif
-            int tl_n = 0;
-#endif
             // The tile coordinates advance incrementally: an integer division per tile sat on the issuer's
             // critical path at every tile boundary.
             int mp = 0, n = 0, ks = 0, z = 0;
             if (tile_begin < tile_end) decode(tile_begin, mp, n, ks, z);
             bool ready = false;  // the next slot's barrier, sampled while the previous slot's MMAs were being issued
             for (int t = tile_begin; t < tile_end && ok; ++t) {
-                GEMM_TL(1);
                 ok = umma::mbar_wait_warp(&tempty[acc], (acc ? acc_phase1 : acc_phase0) ^ 1, abort_flag);
                 if (!ok) break;
-                GEMM_TL(2);
                 if (ARES && mp != cur_mp) {
                     ok = umma::mbar_wait_warp(afull, a_phase, abort_flag);
                     a_phase ^= 1; cur_mp = mp;
                     if (!ok) break;
-                    GEMM_TL(3);
                 }
                 umma::tc_fence_after_sync();
                 const int c_begin = ks * p.chunks_per_split, c_end = min(p.chunks_total, c_begin + p.chunks_per_split);
                 for (int c = c_begin; c < c_end && ok; c += cps) {
                     for (int sl = 0; sl < SLOTS_PER_CHUNK; ++sl) {
-                        GEMM_TL(4);
                         if (!ready) {
                             ok = umma::mbar_wait_warp(&full[stage], phase, abort_flag);
                             if (!ok) break;
                         }
-                        GEMM_TL(5);
                         {   // non-blocking look at the next slot: its latency hides behind this slot's MMAs
                             const int nstage = (stage + 1 == p.stages) ? 0 : stage + 1;
                             ready = __all_sync(0xffffffffu, umma::mbar_test_wait(&full[nstage], nstage ? phase : phase ^ 1));
@@ -725,9 +699,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                     else if (++mp == pairs_m) { mp = 0; if (++ks == p.ksplit) { ks = 0; ++z; } }
                 }
             }
-#ifdef SVDMLP_TIMELINE
-            if (tl_on) { g_gemm_tl[0] = tl_n; g_gemm_tl[1] = tile_end - tile_begin; }
-#endif
         }
     } else if (warp < 2 + kEpiWarps) {  // ---------------- epilogue warps 2..9 (both CTAs, own 128 rows) ----------------
         const int q = warp & 3, half = (warp - 2) >> 2;
@@ -738,20 +709,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
         const bool f16_out = p.out_mode == OUT_F16;
         unsigned char* my_stage = stage_out + (warp - 2) * 4096;
         const uint32_t tempty_leader[2] = {umma::map_to_rank(&tempty[0], 0), umma::map_to_rank(&tempty[1], 0)};
-#ifdef SVDMLP_TIMELINE
-        #if defined(GEMM_TL_DOWN1)
-        const bool tl_on = !ARES && NB == 1 && p.ksplit > 1 && p.K > 4096 && blockIdx.x == 0 && threadIdx.x == 64;
-#elif defined(GEMM_TL_DOWN2)
-        const bool tl_on = NB == 1 && p.resid != nullptr && blockIdx.x == 0 && threadIdx.x == 64;
-#elif defined(GEMM_TL_TS)
-        const bool tl_on = false;
-#elif defined(GEMM_TL_WIDE)
-        const bool tl_on = !ARES && NB == 2 && blockIdx.x == 0 && threadIdx.x == 64;
-#else
-        const bool tl_on = ARES && NB == 2 && blockIdx.x == 0 && threadIdx.x == 64;
-#endif
-        int tl_n = 1020;
-#endif
         // The residual rows this warp will add are requested into L2 one tile ahead (the first tile's at kernel
         // start): read on demand, each 32-column group waited a full HBM round trip inside the epilogue.
         auto prefetch_resid = [&](int tt) {
@@ -768,11 +725,9 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
             int mp, n, ks, z;
             decode(t, mp, n, ks, z);
             const int m = 2 * mp + (int)rank;
-            GEMM_TL(11);
             if (t + 1 < tile_end) prefetch_resid(t + 1);
             ok = umma::mbar_wait_warp(&tfull[acc], acc ? acc_phase1 : acc_phase0, abort_flag);
             if (!ok) break;
-            GEMM_TL(12);
             umma::tc_fence_after_sync();
             const int row = m * BM + q * 32 + lane;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * ACC_COLS;
@@ -842,7 +797,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                         umma::tma_store_2d(&p.tmC, my_stage, col + (int)(z * p.batch_col_off), m * BM + q * 32);
                         umma::bulk_commit();
                     }
-                    GEMM_TL(16);
                 }
             } else if (p.c_tma) {
                 // 16-bit output through shared memory: this warp owns BN/2 columns of its 32 rows; all TMEM
@@ -856,7 +810,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                     umma::tmem_ld32(taddr + c0 + 32, ra[1]);
                     if (NB == 2) umma::tmem_ld32(taddr + BN + c0 + 32, rb[1]);
                     umma::tmem_ld_wait();
-                    GEMM_TL(13);
                     if (c0 == c_last64) release_acc();
                     if (NB == 2 && f16_out) {
 #pragma unroll
@@ -878,9 +831,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                                 packed[hh * 16 + j] = f16_out ? pack_f16(v0, v1) : pack_bf16(v0, v1);
                             }
                     }
-                    GEMM_TL(14);
                     umma::bulk_wait_read0();  // the previous store has finished reading the staging tile
-                    GEMM_TL(15);
                     __syncwarp();
 #pragma unroll
                     for (int ch = 0; ch < 8; ++ch)
@@ -893,7 +844,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                         umma::tma_store_2d(&p.tmC, my_stage, col + (int)(z * p.batch_col_off), m * BM + q * 32);
                         umma::bulk_commit();
                     }
-                    GEMM_TL(16);
                 }
             } else {
                 char* rowbase = reinterpret_cast<char*>(p.C) +
@@ -934,9 +884,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
             if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
             acc = (acc + 1) % NUM_ACC;
         }
-#ifdef SVDMLP_TIMELINE
-        if (tl_on) g_gemm_tl[4095] = tl_n;
-#endif
         if (p.c_tma) umma::bulk_wait_all();
     }
 

@@ -25,7 +25,8 @@ def _case(seed, T, n_in, n_out, r):
 
 def test_noalloc_matches_workspace_entry_point_twice_in_a_row(oracle):
     _gpu.require_gpu()
-    for seed, (T, n_in, n_out, r) in enumerate([(8, 512, 1408, 64), (27, 264, 696, 40)]):
+    # the last case fills the built-in array exactly (32 x 1024 = 32768 values)
+    for seed, (T, n_in, n_out, r) in enumerate([(8, 512, 1408, 64), (27, 264, 696, 40), (32, 512, 704, 1024)]):
         X, U, V = _case(20 + seed, T, n_in, n_out, r)
         Y_ref = binding.svdlinear_forward(X, U, V)
         Y = torch.full((T, n_out), 5.0, dtype=torch.bfloat16, device="cuda")  # caller-owned output
@@ -50,4 +51,12 @@ def test_noalloc_rejects_sizes_beyond_the_fixed_scratch():
                                                   V.data_ptr(), Y.data_ptr(), None)
     too_wide = L.svdlinear_forward_noalloc(X.data_ptr(), 32, 256, 256, 2048, U.data_ptr(), V.data_ptr(), Y.data_ptr(), None)
     assert too_many_tokens == -2 and too_wide == -2
+    # T * r within the array, but the rank's strip of Z would not fit the second kernel's shared memory:
+    # refused on the host, before the clear or any kernel is enqueued (the output stays untouched)
+    Y.fill_(7.0)
+    torch.cuda.synchronize()
+    for T, r in [(4, 8192), (1, 32768), (1, binding.NOALLOC_MAX_R + 8)]:
+        assert L.svdlinear_forward_noalloc(X.data_ptr(), T, 256, 256, r, U.data_ptr(), V.data_ptr(), Y.data_ptr(), None) == -2
+    torch.cuda.synchronize()
+    assert bool((Y == 7.0).all())
     assert "unsupported" in binding.strerror(-2)
