@@ -46,6 +46,7 @@ typedef enum {
 #define SVDMLP_FLAG_NO_CTA_PAIRS 0x80u /* large T: single-CTA tcgen05 kernels only (no cta_group::2 pairs)      */
 #define SVDMLP_FLAG_DECODE_REGISTERS 0x40u /* small T: three register-streaming kernels, not the persistent one */
 #define SVDMLP_FLAG_NO_TMEM_STRIP 0x100u /* large T, ranks <= 256: gate/up with the Z strip in shared memory, not TMEM */
+#define SVDMLP_FLAG_DECODE_COOPERATIVE 0x400u /* small T: cooperative launch of the persistent kernel (residency guaranteed by the driver) instead of a programmatic dependent launch */
 #define SVDMLP_FLAG_NO_WIDE_GATEUP 0x200u /* large T, ranks > 256: gate/up on 128-wide tiles, not 256-wide ones */
 
 /*

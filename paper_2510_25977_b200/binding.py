@@ -22,6 +22,7 @@ FLAG_DECODE_REGISTERS = 0x40
 FLAG_NO_CTA_PAIRS = 0x80
 FLAG_NO_TMEM_STRIP = 0x100
 FLAG_NO_WIDE_GATEUP = 0x200
+FLAG_DECODE_COOPERATIVE = 0x400
 
 EXPORTS = ["svdmlp_create", "svdmlp_forward", "svdmlp_forward_host", "svdmlp_forward_prenorm_residual",
            "svdlinear_forward", "svdlinear_workspace_bytes", "svdlinear_forward_noalloc", "svdmlp_destroy", "svdmlp_strerror",

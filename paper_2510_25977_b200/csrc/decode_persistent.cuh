@@ -1,5 +1,5 @@
-// Decode (T <= 32) path: the whole factored MLP as ONE persistent kernel, one CTA per SM, launched
-// cooperatively.  At small T the MLP is a stream of 6 r (d + ffn) weight bytes through a chain of
+// Decode (T <= 32) path: the whole factored MLP as ONE persistent kernel, one CTA per SM (a
+// programmatic dependent launch; a cooperative launch on request).  At small T the MLP is a stream of 6 r (d + ffn) weight bytes through a chain of
 // three dependent products, so the design goal is that HBM never waits for the chain:
 //
 //  * Create-time packing gives every CTA one contiguous block per phase, already in the order and
@@ -343,6 +343,11 @@ mlp_kernel(const __grid_constant__ Params p) {
         umma::fence_mbar_init();
     }
     __syncthreads();
+    // Programmatic dependent launch: the next kernel in the stream may take this SM as soon as this CTA leaves
+    // it, and this CTA was allowed to start (and set up its barriers) while the tail of the preceding kernel was
+    // still running.  Everything below touches memory that kernel may still use, so wait for it first.
+    umma::pdl_launch_dependents();
+    umma::pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tig = lane & 3;
     const int b = blockIdx.x, nslot = p.nslot;
     const int ksd = s.ksd(), ksr = s.ksr(), zt = s.zt();
@@ -528,6 +533,45 @@ mlp_kernel(const __grid_constant__ Params p) {
                 // zeroed by a select (no branches), even/odd steps use separate accumulators.
                 const int nkb = (ns + 3) >> 2;
                 const unsigned vstride = (unsigned)pa.count * 32u;
+                if (swz) {
+                    // TMA-fed X: d is a multiple of 64, so every column block is whole, and no operand needs
+                    // masking: token rows beyond T and factor rows beyond this CTA's count re-read row 0, which
+                    // only fills accumulator entries that are never stored.  This keeps the loop at a handful of
+                    // address operations per MMA (the masked form below is bound by instruction issue).
+                    const unsigned char* vrow[NTA];
+#pragma unroll
+                    for (int j = 0; j < NTA; ++j) vrow[j] = vs + (8 * j + g < pa.count ? 8 * j + g : 0) * 32 + tig * 8;
+                    const int tsel = ((tig >> 1) << 4) | ((tig & 1) << 3);
+                    for (int kb = warp; kb < nkb; kb += kNW) {
+                        uint2 a[4][MT][2], bv[4][NTA];
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                            for (int hh = 0; hh < 2; ++hh) {
+                                if (mt * 16 + hh * 8 < ROWS) {
+                                    const int row = mt * 16 + hh * 8 + g;
+                                    const int rr = (kb0 + kb) * s.T + (row < s.T ? row : 0), sw = (rr & 7) << 4;
+                                    const unsigned char* xb = xs + (rr << 7);
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) a[e][mt][hh] = lds64(xb + ((2 * e * 16 + tsel) ^ sw));
+                                } else {
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) a[e][mt][hh] = make_uint2(0, 0);
+                                }
+                            }
+#pragma unroll
+                        for (int j = 0; j < NTA; ++j)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) bv[e][j] = lds64(vrow[j] + (unsigned)(kb * 4 + e) * vstride);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+#pragma unroll
+                            for (int j = 0; j < NTA; ++j)
+#pragma unroll
+                                for (int mt = 0; mt < MT; ++mt)
+                                    mma_bf16(acc[e & 1][mt][j], a[e][mt][0].x, a[e][mt][1].x, a[e][mt][0].y, a[e][mt][1].y, bv[e][j].x, bv[e][j].y);
+                    }
+                } else
                 for (int kb = warp; kb < nkb; kb += kNW) {
                     const int stb = kb * 4;  // first step of the block within the group
                     uint2 a[4][MT][2], bv[4][NTA];

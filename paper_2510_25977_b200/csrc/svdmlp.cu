@@ -499,10 +499,19 @@ int persist_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp3
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(h->persist_grid); cfg.blockDim = dim3(dpersist::kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = s;
-    // Cooperative: all CTAs must be resident at once (they wait on one another).
+    // The CTAs wait on one another, so all of them must become resident: one CTA per SM and a grid of at most
+    // the SM count.  Default: programmatic dependent launch (a CTA starts on an SM as soon as the preceding
+    // kernel's CTA has left it and orders itself behind that kernel with griddepcontrol.wait; 0.6 us per step
+    // less than a cooperative launch, which drains the GPU first).  SVDMLP_FLAG_DECODE_COOPERATIVE asks for the
+    // cooperative launch, whose residency the driver guarantees even when other work shares the GPU.
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
+    if (h->flags & SVDMLP_FLAG_DECODE_COOPERATIVE) {
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+    } else {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+    }
     cfg.attrs = attr; cfg.numAttrs = 1;
     {
         ProfScope ps(h, "mlp_decode", s);
