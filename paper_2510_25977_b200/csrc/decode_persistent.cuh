@@ -1,6 +1,7 @@
 // Decode (T <= 32) path: the whole factored MLP as ONE persistent kernel, one CTA per SM (a
-// programmatic dependent launch; a cooperative launch on request).  At small T the MLP is a stream of 6 r (d + ffn) weight bytes through a chain of
-// three dependent products, so the design goal is that HBM never waits for the chain:
+// programmatic dependent launch; a cooperative launch on request).  At small T the MLP is a stream
+// of 6 r (d + ffn) weight bytes through a chain of three dependent products, so the design goal is
+// that HBM never waits for the chain:
 //
 //  * Create-time packing gives every CTA one contiguous block per phase, already in the order and
 //    layout its warps consume, so the producer warp moves it with a few large 1-D bulk copies into a

@@ -182,3 +182,16 @@ def sample_rows(T: int, tile: int = 128, max_rows: int = 64) -> list[int]:
         rows.update({lo, hi, (lo + hi) // 2, min(hi, lo + 37)})
     rows = sorted(r for r in rows if 0 <= r < T)
     return rows[:max_rows]
+
+
+def rows_of_every_tile(T: int, tile: int = 128, per_tile: int = 2) -> list[int]:
+    """Token rows for sampled parity at the largest T: `per_tile` rows of EVERY `tile`-row tile (a position
+    that moves from tile to tile, plus the tile's last row), so that a fault tied to the n-th tile a
+    persistent CTA walks cannot hide between samples."""
+    rows = set()
+    for m in range((T + tile - 1) // tile):
+        lo, hi = m * tile, min(T, (m + 1) * tile) - 1
+        rows.add(hi)
+        for j in range(per_tile - 1):
+            rows.add(lo + (m * 37 + j * 53) % (hi - lo + 1))
+    return sorted(rows)

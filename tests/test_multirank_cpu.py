@@ -38,6 +38,14 @@ def _worker(rank, world, port, out_dir):
     lo, hi = sharding.shard_rows(T, world, rank)
     Y_local = oracle.svdmlp(X[lo:hi], *f.tensors())       # the single-device forward on this rank's rows
     slowest = sharding.max_over_ranks(10.0 + rank, dist)  # timing reduction: max over ranks
+    import bench   # the benchmark's own rank logic: row blocks of one world * T batch at large T, replicas at decode
+    assert bench.local_tokens(1024, world, rank, "tensor") == 1024
+    blo, bhi = sharding.shard_rows(world * 300, world, rank)
+    assert bench.local_tokens(300, world, rank, "tensor") == bhi - blo
+    assert bench.local_tokens(8, world, rank, "skinny") == 8
+    total = torch.tensor([bench.local_tokens(300, world, rank, "tensor")])
+    dist.all_reduce(total)
+    assert int(total) == world * 300   # the blocks of all ranks add up to the whole batch
     np.save(os.path.join(out_dir, f"y{rank}.npy"), Y_local)
     np.save(os.path.join(out_dir, f"t{rank}.npy"), np.array([slowest, lo, hi]))
     dist.barrier()
@@ -57,3 +65,18 @@ def test_two_ranks_shard_rows_and_reduce_time(tmp_path, oracle):
         slowest, lo, hi = np.load(tmp_path / f"t{k}.npy")
         assert slowest == 11.0
         assert (lo, hi) == sharding.shard_rows(T, world, k)
+
+
+def test_bench_gpus_flag_spawns_one_rank_per_gpu():
+    """`bench.py --gpus 2` started as a plain process re-launches itself as two ranks (here the reference arm, which
+    needs no GPU: rank 0 prints the one JSON line, rank 1 exits 0 without work)."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--steps", "1",
+                          "--warmup", "0"], capture_output=True, text=True, timeout=900, cwd=ROOT, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    j = json.loads(lines[0])
+    assert j["impl"] == "reference" and j["n_gpus"] == 2 and j["value"] > 0
