@@ -47,6 +47,7 @@ typedef enum {
 #define SVDMLP_FLAG_DECODE_REGISTERS 0x40u /* small T: three register-streaming kernels, not the persistent one */
 #define SVDMLP_FLAG_NO_TMEM_STRIP 0x100u /* large T, ranks <= 256: gate/up with the Z strip in shared memory, not TMEM */
 #define SVDMLP_FLAG_DECODE_COOPERATIVE 0x400u /* small T: cooperative launch of the persistent kernel (residency guaranteed by the driver) instead of a programmatic dependent launch */
+#define SVDMLP_FLAG_TOKEN_SLABS 0x800u /* large T: gate/up and the first down product run over token slabs whose H (64 MB) stays in L2; off by default (slower as measured) */
 #define SVDMLP_FLAG_NO_WIDE_GATEUP 0x200u /* large T, ranks > 256: gate/up on 128-wide tiles, not 256-wide ones */
 
 /*
@@ -106,6 +107,24 @@ int svdmlp_forward_prenorm_residual(svdmlp_t* h, const float* h_in, float* h_out
 int svdlinear_forward(const void* X, int T, int in, int out, int r, const void* U, const void* V,
                       void* Y, void* workspace, size_t workspace_bytes, void* stream);
 size_t svdlinear_workspace_bytes(int T, int in, int out, int r);
+
+/*
+ * The same operator with a handle (Section 4.2.1; the factors of a layer are fixed at inference time, Section
+ * 2.1): svdlinear_create does once what svdlinear_forward repeats on every call for T > 32 - the fp16 re-encoding
+ * of U that the second product needs (its first operand, Z, is fp16) and the tensor maps of the factors - and owns
+ * the workspace, sized for max_T.  The handle borrows U and V (they must outlive it).  svdlinear_apply computes
+ * Y[T, out] = (X V^T) U^T for 1 <= T <= max_T, asynchronously on `stream`.
+ * Number range for T > 32 (both entry points): Z = X V^T and the re-encoded U are fp16, so |Z| and |U| must stay
+ * below 65504; svdlinear_create checks U and, if a value exceeds the range, svdlinear_apply returns
+ * SVDMLP_ERR_UNSUPPORTED for T > 32 (T <= 32 runs on bf16 kernels with fp32 intermediates and has no such limit).
+ * svdlinear_forward cannot report the condition (it never synchronises): out-of-range factors give inf/NaN there.
+ * Errors: INVALID_ARG, ALIGNMENT, ARCH, NOMEM, CUDA, UNSUPPORTED.
+ */
+typedef struct svdlinear svdlinear_t; /* opaque */
+int svdlinear_create(svdlinear_t** out_handle, int in, int out, int r, const void* U, const void* V, int max_T,
+                     void* stream);
+int svdlinear_apply(svdlinear_t* h, const void* X, int T, void* Y, void* stream);
+int svdlinear_destroy(svdlinear_t* h);
 
 /*
  * XUV operator without any allocation (the paper has no counterpart: it is a packaging variant

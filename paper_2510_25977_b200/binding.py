@@ -23,9 +23,11 @@ FLAG_NO_CTA_PAIRS = 0x80
 FLAG_NO_TMEM_STRIP = 0x100
 FLAG_NO_WIDE_GATEUP = 0x200
 FLAG_DECODE_COOPERATIVE = 0x400
+FLAG_TOKEN_SLABS = 0x800
 
 EXPORTS = ["svdmlp_create", "svdmlp_forward", "svdmlp_forward_host", "svdmlp_forward_prenorm_residual",
-           "svdlinear_forward", "svdlinear_workspace_bytes", "svdlinear_forward_noalloc", "svdmlp_destroy", "svdmlp_strerror",
+           "svdlinear_forward", "svdlinear_workspace_bytes", "svdlinear_forward_noalloc",
+           "svdlinear_create", "svdlinear_apply", "svdlinear_destroy", "svdmlp_destroy", "svdmlp_strerror",
            "svdmlp_last_device_status", "svdmlp_launch_count", "svdmlp_path_name",
            "svdmlp_profile_enable", "svdmlp_profile_read", "svdmlp_profile_name", "svdmlp_stage_mask",
            "svdmlp_block_aligned_rank", "svdmlp_selftest_timeout"]
@@ -59,6 +61,12 @@ def lib() -> ctypes.CDLL:
         L.svdlinear_forward.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.svdlinear_forward_noalloc.restype = ci
         L.svdlinear_forward_noalloc.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp]
+        L.svdlinear_create.restype = ci
+        L.svdlinear_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, vp, vp, ci, vp]
+        L.svdlinear_apply.restype = ci
+        L.svdlinear_apply.argtypes = [vp, vp, ci, vp, vp]
+        L.svdlinear_destroy.restype = ci
+        L.svdlinear_destroy.argtypes = [vp]
         L.svdlinear_workspace_bytes.restype = ctypes.c_size_t
         L.svdlinear_workspace_bytes.argtypes = [ci, ci, ci, ci]
         L.svdmlp_destroy.restype = ci
@@ -192,6 +200,43 @@ def svdlinear_forward(X, U, V, Y=None, workspace=None, stream=None) -> torch.Ten
     _check(lib().svdlinear_forward(_ptr(X), T, n_in, n_out, r, _ptr(U), _ptr(V), _ptr(Y), _ptr(workspace),
                                    workspace.numel(), _stream(stream)), "svdlinear_forward")
     return Y
+
+
+class LinearHandle:
+    """Owns one svdlinear_t and keeps U and V alive (the library borrows their memory)."""
+
+    def __init__(self, ptr, keep, n_out):
+        self.ptr, self._keep, self.n_out = ptr, keep, n_out
+
+    def close(self):
+        if self.ptr:
+            lib().svdlinear_destroy(self.ptr)
+            self.ptr = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def svdlinear_create(U, V, max_T: int, stream=None) -> LinearHandle:
+    n_out, r = U.shape
+    n_in = V.shape[1]
+    h = ctypes.c_void_p()
+    _check(lib().svdlinear_create(ctypes.byref(h), n_in, n_out, r, _ptr(U), _ptr(V), max_T, _stream(stream)), "svdlinear_create")
+    return LinearHandle(h, (U, V), n_out)
+
+
+def svdlinear_apply(h: LinearHandle, X, Y=None, stream=None) -> torch.Tensor:
+    if Y is None:
+        Y = torch.empty((X.shape[0], h.n_out), dtype=torch.bfloat16, device=X.device)
+    _check(lib().svdlinear_apply(h.ptr, _ptr(X), X.shape[0], _ptr(Y), _stream(stream)), "svdlinear_apply")
+    return Y
+
+
+def svdlinear_destroy(h: LinearHandle):
+    h.close()
 
 
 NOALLOC_MAX_T = 32

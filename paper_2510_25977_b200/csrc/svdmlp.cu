@@ -260,7 +260,7 @@ int down1_tile_width(int rd) {
 // Fill the shape-dependent part of a plan (tensor maps are set by the caller).
 // want_res: keep the A strip resident if it fits.  allow_split: use split-K to fill the machine.
 void plan_gemm(GemmPlan& g, int nb, int bn, bool want_res, bool allow_split, int M, int N, int K, int batch,
-               bool c_tma = false, bool want_pair = false) {
+               bool c_tma = false, bool want_pair = false, int force_ksplit = 0) {
     using namespace tensorpath;
     g.nb = nb; g.bn = bn; g.pair = false;
     GemmParams& p = g.p;
@@ -289,7 +289,7 @@ void plan_gemm(GemmPlan& g, int nb, int bn, bool want_res, bool allow_split, int
         int ks = std::max(1, units / std::max(1, base_tiles));
         ks = std::min(ks, std::max(1, p.chunks_total / 8));  // keep at least 8 chunks per split
         ks = std::min(ks, 16);
-        p.ksplit = ks;
+        p.ksplit = force_ksplit > 0 ? force_ksplit : ks;   // forced: token slabs of one forward share one partial layout
     }
     p.chunks_per_split = (p.chunks_total + p.ksplit - 1) / p.ksplit;
     p.ksplit = (p.chunks_total + p.chunks_per_split - 1) / p.chunks_per_split;  // no empty split
@@ -319,6 +319,15 @@ void plan_gemm(GemmPlan& g, int nb, int bn, bool want_res, bool allow_split, int
 
 }  // namespace
 
+// Token slabs: gate/up and the first half of the down chain run slab by slab so that a slab's H is read back while
+// it is still in L2.  Each slab has its own tensor maps (the same buffers, offset by the slab's first row).
+struct SlabMaps { CUtensorMap zg, zu, hc, h; };
+constexpr int kMaxSlabs = 32;
+struct SlabPlan {
+    int T, rows, n;   // T the plan was made for (0: none), rows per slab (a multiple of 256), number of slabs
+    SlabMaps maps[kMaxSlabs];
+};
+
 struct svdmlp {
     int d, ffn, rg, ru, rd, max_T;
     unsigned flags;
@@ -346,6 +355,7 @@ struct svdmlp {
     // cached X map and output maps of the TMA-store epilogues (box [32 rows, 64 columns])
     const void* x_ptr; int x_T; CUtensorMap mX;
     CUtensorMap mHc, mYc; const void* y_ptr; int y_T, y_f32;
+    SlabPlan slabs;                   // token slabs of the gate/up -> down-1 pair for the last T seen (maps cached)
     CUtensorMap mUg64, mUu64, mUd64;  // half-tile boxes [64 rows, 64 columns] for the CTA-pair kernels
     CUtensorMap mVg64, mVu64, mVg128, mVu128, mVdHalf;  // half-tile boxes of the first-GEMM factors
     // persistent decode kernel: cached tensor map of X, packed factors (owned), intermediates and barrier words
@@ -596,6 +606,38 @@ int launch_reduce(const float* part, int ksplit, long split_stride, long n, __ha
     return SVDMLP_OK;
 }
 
+// H bytes one slab may hold with SVDMLP_FLAG_TOKEN_SLABS: inside the 126 MB L2 next to the factors, Z and the
+// split-K partials.  Without the flag the two kernels run over all T rows at once: measured on B200, every slab
+// boundary (two more launches, fewer tiles per wave, deeper split-K) costs more than the HBM traffic of H it
+// saves (config 4, r = 128, T = 8192: 159 us unslabbed, 192 / 202 / 232 us with 64 / 48 / 32 MB slabs).
+constexpr size_t kSlabBytes = (size_t)64 << 20;
+
+const SlabPlan* slab_plan(svdmlp* h, int T) {
+    SlabPlan& sp = h->slabs;
+    if (sp.T == T) return &sp;
+    const size_t row_bytes = (size_t)h->ffn * 2;
+    int n = 1;
+    if ((h->flags & SVDMLP_FLAG_TOKEN_SLABS) && (size_t)T * row_bytes > kSlabBytes + kSlabBytes / 2)
+        n = (int)(((size_t)T * row_bytes + kSlabBytes - 1) / kSlabBytes);
+    n = std::min(n, kMaxSlabs);
+    int rows = ((T + n - 1) / n + 255) / 256 * 256;   // whole CTA-pair row strips
+    n = (T + rows - 1) / rows;
+    const int R = h->rg + h->ru;
+    for (int i = 0; i < n; ++i) {
+        const int row0 = i * rows, Ts = std::min(rows, T - row0);
+        SlabMaps& m = sp.maps[i];
+        if (make_map(&m.zg, h->Z16 + (size_t)row0 * R, Ts, h->rg, R, 128) != SVDMLP_OK ||
+            make_map(&m.zu, h->Z16 + (size_t)row0 * R + h->rg, Ts, h->ru, R, 128) != SVDMLP_OK ||
+            make_map(&m.hc, h->H16 + (size_t)row0 * h->ffn, Ts, h->ffn, h->ffn, 32) != SVDMLP_OK ||
+            make_map(&m.h, h->H16 + (size_t)row0 * h->ffn, Ts, h->ffn, h->ffn, 128) != SVDMLP_OK) {
+            sp.T = 0;
+            return nullptr;
+        }
+    }
+    sp.T = T; sp.rows = rows; sp.n = n;
+    return &sp;
+}
+
 int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32, const float* resid, cudaStream_t s) {
     using namespace tensorpath;
     if (!h->tensor_ok) return SVDMLP_ERR_UNSUPPORTED;
@@ -633,13 +675,23 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     }
     }
     // 2. H = SiLU(Zg Ug^T) .* (Zu Uu^T)   (phase 2 of Algorithm 3 with its epilogue), fp16 out
+    // 3. Zd = H Vd^T   (phase 1 of the down-projection XUV chain), split-K fp32 partials -> fp16
+    // On request (SVDMLP_FLAG_TOKEN_SLABS) the two run slab by slab over the token rows when H as a whole would
+    // not stay in L2 between its one write and its one read (the analogue of the paper's row-strip loop,
+    // Section 4.2.1): a slab's H is produced and consumed while it is still cache-resident.
+    const SlabPlan* sp = slab_plan(h, T);
+    if (sp == nullptr) return SVDMLP_ERR_CUDA;
+    int down1_ksplit = 0;
+    for (int si = 0; si < sp->n; ++si) {
+    const int row0 = si * sp->rows, Ts = std::min(sp->rows, T - row0);
+    const SlabMaps& sm = sp->maps[si];
     if (mask & 2u) {
-    plan_gemm(g, 2, 128, true, false, T, h->ffn, h->rg, 1, true, !(h->flags & SVDMLP_FLAG_NO_CTA_PAIRS));
-    g.p.tmC = h->mHc;
-    g.p.tmA[0] = h->mZg; g.p.tmA[1] = h->mZu;
+    plan_gemm(g, 2, 128, true, false, Ts, h->ffn, h->rg, 1, true, !(h->flags & SVDMLP_FLAG_NO_CTA_PAIRS));
+    g.p.tmC = sm.hc;
+    g.p.tmA[0] = sm.zg; g.p.tmA[1] = sm.zu;
     g.p.tmB[0] = g.pair ? h->mUg64 : h->mUg; g.p.tmB[1] = g.pair ? h->mUu64 : h->mUu;
     g.p.a_fmt = umma::kFmtF16; g.p.b_fmt = umma::kFmtF16; g.p.status = h->status_dev;
-    g.p.C = h->H16; g.p.ldc = h->ffn; g.p.out_mode = OUT_F16;
+    g.p.C = h->H16 + (size_t)row0 * h->ffn; g.p.ldc = h->ffn; g.p.out_mode = OUT_F16;
     // ranks up to 256 on CTA pairs: the Z strip lives in tensor memory and the branches run one after the other
     const bool ts = g.pair && g.ares && h->rg == h->ru && h->rg <= 256 && !(h->flags & SVDMLP_FLAG_NO_TMEM_STRIP);
     if (ts) {
@@ -664,20 +716,25 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     if (rc != SVDMLP_OK) return rc;
     h->launches += 1;
     }
-    // 3. Zd = H Vd^T   (phase 1 of the down-projection XUV chain), split-K fp32 partials -> fp16
     if (mask & 4u) {
     const int bn3 = down1_tile_width(h->rd);
-    plan_gemm(g, 1, bn3, false, true, T, h->rd, h->ffn, 1, false, pairs_ok);
-    g.p.tmA[0] = h->mH; g.p.tmA[1] = h->mH;
+    plan_gemm(g, 1, bn3, false, true, Ts, h->rd, h->ffn, 1, false, pairs_ok, down1_ksplit);
+    if (si == 0) down1_ksplit = g.p.ksplit;
+    if (g.p.ksplit != down1_ksplit) return SVDMLP_ERR_UNSUPPORTED;  // cannot happen: the split depends on K alone once forced
+    g.p.tmA[0] = sm.h; g.p.tmA[1] = sm.h;
     g.p.tmB[0] = g.pair ? h->mVdHalf : h->mVd; g.p.tmB[1] = g.p.tmB[0];
     g.p.a_fmt = umma::kFmtF16; g.p.b_fmt = umma::kFmtF16; g.p.status = h->status_dev;
     if ((size_t)g.p.ksplit * T * h->rd > h->part_elems) return SVDMLP_ERR_NOMEM;
-    g.p.C = h->part; g.p.ldc = h->rd; g.p.split_stride = (long)T * h->rd; g.p.out_mode = OUT_F32;
+    g.p.C = h->part + (size_t)row0 * h->rd; g.p.ldc = h->rd; g.p.split_stride = (long)T * h->rd; g.p.out_mode = OUT_F32;
     { ProfScope ps(h, "down1", s); rc = launch_gemm(g, s); }
     if (rc != SVDMLP_OK) return rc;
-    { ProfScope ps(h, "down1_reduce", s); rc = launch_reduce(h->part, g.p.ksplit, (long)T * h->rd, (long)T * h->rd, h->Zd16, s); }
+    h->launches += 1;
+    }
+    }
+    if (mask & 4u) {
+    { ProfScope ps(h, "down1_reduce", s); rc = launch_reduce(h->part, down1_ksplit, (long)T * h->rd, (long)T * h->rd, h->Zd16, s); }
     if (rc != SVDMLP_OK) return rc;
-    h->launches += 2;
+    h->launches += 1;
     }
     // 4. Y = Zd Ud^T   (phase 2 of the XUV chain)
     if (mask & 8u) {
@@ -1128,6 +1185,49 @@ extern "C" int svdlinear_forward_noalloc(const void* X, int T, int in, int out, 
     return SVDMLP_OK;
 }
 
+struct svdlinear {
+    int in, out, r, max_T;
+    const void *U, *V;
+    void* ws; size_t ws_bytes;
+    float* f32; __half *z16, *u16;
+    bool u16_ok;
+    CUtensorMap mV, mU, mZ, mZc;
+    const void* x_ptr; int x_T; CUtensorMap mX;
+    const void* y_ptr; int y_T; CUtensorMap mYc;
+};
+
+namespace {
+// The two products of the XUV operator on the tcgen05 kernels.  Both stream their operands; with at least two
+// token tiles they run on CTA pairs (cta_group::2, 256 x 256 tiles, each CTA loading half of the B tile) and
+// leave through TMA stores.  Z[T, r] passes through global memory in fp16 (L2-resident at these sizes).
+int lin_tensor_run(const CUtensorMap& mX, const CUtensorMap& mV, const CUtensorMap& mU, const CUtensorMap& mZ,
+                   const CUtensorMap& mZc, const CUtensorMap& mYc, float* f32, __half* z16, void* Y, int T, int in,
+                   int out, int r, cudaStream_t s) {
+    using namespace tensorpath;
+    int rc;
+    const bool pr = T > BM;
+    const int bn = pr ? 256 : 128;
+    GemmPlan g;
+    plan_gemm(g, 1, bn, false, true, T, r, in, 1, true, pr);
+    g.p.tmA[0] = mX; g.p.tmA[1] = mX; g.p.tmB[0] = mV; g.p.tmB[1] = mV; g.p.tmC = mZc;
+    g.p.a_fmt = umma::kFmtBF16; g.p.b_fmt = umma::kFmtBF16; g.p.status = nullptr;
+    if (g.p.ksplit > 1) {
+        g.p.c_tma = 0;  // fp32 partials are stored directly
+        g.p.C = f32; g.p.ldc = r; g.p.split_stride = (long)T * r; g.p.out_mode = OUT_F32;
+        if ((rc = launch_gemm(g, s)) != SVDMLP_OK) return rc;
+        if ((rc = launch_reduce(f32, g.p.ksplit, (long)T * r, (long)T * r, z16, s)) != SVDMLP_OK) return rc;
+    } else {
+        g.p.C = z16; g.p.ldc = r; g.p.out_mode = OUT_F16;
+        if ((rc = launch_gemm(g, s)) != SVDMLP_OK) return rc;
+    }
+    plan_gemm(g, 1, bn, false, false, T, out, r, 1, true, pr);
+    g.p.tmA[0] = mZ; g.p.tmA[1] = mZ; g.p.tmB[0] = mU; g.p.tmB[1] = mU; g.p.tmC = mYc;
+    g.p.a_fmt = umma::kFmtF16; g.p.b_fmt = umma::kFmtF16; g.p.status = nullptr;
+    g.p.C = Y; g.p.ldc = out; g.p.out_mode = OUT_BF16;
+    return launch_gemm(g, s);
+}
+}  // namespace
+
 extern "C" {
 
 // ---- XUV operator --------------------------------------------------------------------------------
@@ -1188,31 +1288,76 @@ int svdlinear_forward(const void* X, int T, int in, int out, int r, const void* 
     if ((rc = launch_convert(U, u16, (long)out * r, flag, s)) != SVDMLP_OK) return rc;
     if ((rc = make_map(&mU, u16, out, r, r, 128)) != SVDMLP_OK) return rc;
     if ((rc = make_map(&mZ, z16, T, r, r, 128)) != SVDMLP_OK) return rc;
-    // Both products stream their operands; with at least two token tiles they run on CTA pairs (cta_group::2,
-    // 256 x 256 tiles, each CTA loading half of the B tile) and leave through TMA stores.
-    const bool pr = T > BM;
-    const int bn = pr ? 256 : 128;
     CUtensorMap mZc, mYc;
     if ((rc = make_map(&mZc, z16, T, r, r, 32)) != SVDMLP_OK) return rc;
     if ((rc = make_map(&mYc, Y, T, out, out, 32)) != SVDMLP_OK) return rc;
-    GemmPlan g;
-    plan_gemm(g, 1, bn, false, true, T, r, in, 1, true, pr);
-    g.p.tmA[0] = mX; g.p.tmA[1] = mX; g.p.tmB[0] = mV; g.p.tmB[1] = mV; g.p.tmC = mZc;
-    g.p.a_fmt = umma::kFmtBF16; g.p.b_fmt = umma::kFmtBF16; g.p.status = nullptr;
-    if (g.p.ksplit > 1) {
-        g.p.c_tma = 0;  // fp32 partials are stored directly
-        g.p.C = f32; g.p.ldc = r; g.p.split_stride = (long)T * r; g.p.out_mode = OUT_F32;
-        if ((rc = launch_gemm(g, s)) != SVDMLP_OK) return rc;
-        if ((rc = launch_reduce(f32, g.p.ksplit, (long)T * r, (long)T * r, z16, s)) != SVDMLP_OK) return rc;
-    } else {
-        g.p.C = z16; g.p.ldc = r; g.p.out_mode = OUT_F16;
-        if ((rc = launch_gemm(g, s)) != SVDMLP_OK) return rc;
+    return lin_tensor_run(mX, mV, mU, mZ, mZc, mYc, f32, z16, Y, T, in, out, r, s);
+}
+
+// ---- XUV operator with a handle: everything that does not depend on the call is done once ---------------
+int svdlinear_create(svdlinear_t** out_h, int in, int out, int r, const void* U, const void* V, int max_T, void* stream) {
+    if (out_h == nullptr) return SVDMLP_ERR_INVALID_ARG;
+    *out_h = nullptr;
+    if (!U || !V || in <= 0 || out <= 0 || r <= 0 || max_T <= 0) return SVDMLP_ERR_INVALID_ARG;
+    if ((in | out | r) & 7) return SVDMLP_ERR_ALIGNMENT;
+    if (!aligned16(U) || !aligned16(V)) return SVDMLP_ERR_ALIGNMENT;
+    int rc = check_arch();
+    if (rc != SVDMLP_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    svdlinear* h = new (std::nothrow) svdlinear();
+    if (h == nullptr) return SVDMLP_ERR_NOMEM;
+    memset(h, 0, sizeof(*h));
+    h->in = in; h->out = out; h->r = r; h->max_T = max_T; h->U = U; h->V = V;
+    h->ws_bytes = svdlinear_workspace_bytes(max_T, in, out, r);
+    if (cudaMalloc(&h->ws, h->ws_bytes) != cudaSuccess) { cudaGetLastError(); delete h; return SVDMLP_ERR_NOMEM; }
+    h->f32 = reinterpret_cast<float*>(h->ws);
+    h->z16 = reinterpret_cast<__half*>(reinterpret_cast<char*>(h->ws) + ((lin_f32_elems(max_T, r) * 4 + 255) & ~(size_t)255));
+    h->u16 = h->z16 + (((size_t)max_T * r * 2 + 255) & ~(size_t)255) / 2;
+    int* flag = reinterpret_cast<int*>(h->u16 + (((size_t)out * r * 2 + 255) & ~(size_t)255) / 2);
+    int over = 0;
+    bool ok = cudaMemsetAsync(flag, 0, sizeof(int), s) == cudaSuccess &&
+              launch_convert(U, h->u16, (long)out * r, flag, s) == SVDMLP_OK &&
+              cudaMemcpyAsync(&over, flag, sizeof(int), cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+              cudaStreamSynchronize(s) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); svdlinear_destroy(h); return SVDMLP_ERR_CUDA; }
+    h->u16_ok = over == 0;   // a value of U beyond the fp16 range: only the small-T (bf16) kernels can be used
+    if (h->u16_ok && max_T > kSkinnyMaxT) {
+        rc = make_map(&h->mV, V, r, in, in, 128);
+        if (rc == SVDMLP_OK) rc = make_map(&h->mU, h->u16, out, r, r, 128);
+        if (rc == SVDMLP_OK) rc = make_map(&h->mZ, h->z16, max_T, r, r, 128);
+        if (rc == SVDMLP_OK) rc = make_map(&h->mZc, h->z16, max_T, r, r, 32);
+        if (rc != SVDMLP_OK) { svdlinear_destroy(h); return rc; }
     }
-    plan_gemm(g, 1, bn, false, false, T, out, r, 1, true, pr);
-    g.p.tmA[0] = mZ; g.p.tmA[1] = mZ; g.p.tmB[0] = mU; g.p.tmB[1] = mU; g.p.tmC = mYc;
-    g.p.a_fmt = umma::kFmtF16; g.p.b_fmt = umma::kFmtF16; g.p.status = nullptr;
-    g.p.C = Y; g.p.ldc = out; g.p.out_mode = OUT_BF16;
-    return launch_gemm(g, s);
+    *out_h = h;
+    return SVDMLP_OK;
+}
+
+int svdlinear_apply(svdlinear_t* h, const void* X, int T, void* Y, void* stream) {
+    if (h == nullptr || X == nullptr || Y == nullptr || T <= 0 || T > h->max_T) return SVDMLP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Y)) return SVDMLP_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (T <= kSkinnyMaxT)   // weight-streaming kernels read the bf16 factors as they are
+        return svdlinear_forward(X, T, h->in, h->out, h->r, h->U, h->V, Y, h->ws, h->ws_bytes, stream);
+    if (!h->u16_ok) return SVDMLP_ERR_UNSUPPORTED;
+    int rc;
+    if (h->x_ptr != X || h->x_T != T) {
+        if ((rc = make_map(&h->mX, X, T, h->in, h->in, tensorpath::BM)) != SVDMLP_OK) return rc;
+        h->x_ptr = X; h->x_T = T;
+    }
+    if (h->y_ptr != Y || h->y_T != T) {
+        if ((rc = make_map(&h->mYc, Y, T, h->out, h->out, 32)) != SVDMLP_OK) return rc;
+        h->y_ptr = Y; h->y_T = T;
+    }
+    return lin_tensor_run(h->mX, h->mV, h->mU, h->mZ, h->mZc, h->mYc, h->f32, h->z16, Y, T, h->in, h->out, h->r, s);
+}
+
+int svdlinear_destroy(svdlinear_t* h) {
+    if (h == nullptr) return SVDMLP_OK;
+    cudaDeviceSynchronize();
+    cudaGetLastError();
+    if (h->ws != nullptr) cudaFree(h->ws);
+    delete h;
+    return SVDMLP_OK;
 }
 
 }  // extern "C"

@@ -345,3 +345,48 @@ def test_svdlinear_xuv_operator(oracle, T, n_in, n_out, r):
     rows = inputs.sample_rows(T, max_rows=32 if r <= 256 else 10)
     # bf16 output rounding alone costs ~1.4e-3 mean relative error
     _gpu.assert_close(Y[rows], oracle.svdlinear(X[rows], U, V), f"svdlinear T={T}")
+
+
+def test_token_slab_schedule(oracle):
+    """Gate/up and the first down product slab by slab over the tokens (three ragged slabs here: 5000 rows of
+    ffn = 14336 are 143 MB of H): same result as the oracle, two rows of every 128-row tile compared."""
+    T = 5000
+    f = inputs.direct_factors(4096, 14336, 128, seed=0, device="cuda")
+    X = inputs.activations(T, 4096, seed=2, device="cuda")
+    Y = _gpu.run_mlp(f, X, flags=binding.FLAG_TOKEN_SLABS)
+    rows = inputs.rows_of_every_tile(T, per_tile=2)
+    _gpu.assert_close(Y[rows], _gpu.oracle_rows(oracle, f, X, rows), "token slabs")
+
+
+@pytest.mark.parametrize("T,n_in,n_out,r", [(5, 264, 696, 40), (300, 264, 696, 40), (1024, 2048, 4096, 256)])
+def test_svdlinear_handle(oracle, T, n_in, n_out, r):
+    """svdlinear_create / svdlinear_apply: same operator, U re-encoded and maps built once; several T per handle."""
+    V = inputs.normal_tensor(12, 0, (r, n_in), scale=n_in ** -0.5, device="cuda")
+    U = inputs.normal_tensor(12, 1, (n_out, r), scale=r ** -0.5, device="cuda")
+    h = binding.svdlinear_create(U, V, max_T=max(T, 64))
+    for t in (T, min(T, 40), T):
+        X = inputs.activations(t, n_in, seed=12 + t, device="cuda")
+        Y = binding.svdlinear_apply(h, X)
+        torch.cuda.synchronize()
+        rows = inputs.sample_rows(t, max_rows=32)
+        _gpu.assert_close(Y[rows], oracle.svdlinear(X[rows], U, V), f"svdlinear handle T={t}")
+    with pytest.raises(binding.SvdMlpError):
+        binding.svdlinear_apply(h, inputs.activations(max(T, 64) + 1, n_in, device="cuda"))
+    binding.svdlinear_destroy(h)
+
+
+def test_svdlinear_handle_reports_factors_outside_the_fp16_range():
+    """A factor value beyond 65504 cannot be re-encoded for the large-T kernels: the handle says so (status -2) for
+    T > 32 instead of returning inf/NaN, and still serves small T on the bf16 kernels."""
+    V = inputs.normal_tensor(13, 0, (32, 256), scale=256 ** -0.5, device="cuda")
+    U = inputs.normal_tensor(13, 1, (512, 32), scale=32 ** -0.5, device="cuda").clone()
+    U[3, 5] = 1.0e5
+    h = binding.svdlinear_create(U, V, max_T=128)
+    X = inputs.activations(128, 256, seed=13, device="cuda")
+    with pytest.raises(binding.SvdMlpError) as e:
+        binding.svdlinear_apply(h, X)
+    assert e.value.status == -2
+    Y = binding.svdlinear_apply(h, X[:8].contiguous())
+    torch.cuda.synchronize()
+    assert torch.isfinite(Y.float()).all()
+    binding.svdlinear_destroy(h)
