@@ -99,6 +99,24 @@ int svdmlp_forward_prenorm_residual(svdmlp_t* h, const float* h_in, float* h_out
                                     float eps, void* stream);
 
 /*
+ * The two halves of the forward pass for tensor parallelism over ffn (Section 4.2.2, last paragraph, and
+ * Figure 4: gate and up projections partitioned by columns, the down projection by rows, one all-reduce).  With
+ * factored weights the partition falls on the rank-r chain: shard g of G holds the rows Ug[F_g, :], Uu[F_g, :]
+ * and the columns Vd[:, F_g] of its slice F_g of ffn (as contiguous arrays; a handle is created on them with
+ * ffn = |F_g|), and Vg, Vu, Ud whole.  Then  Zd = sum_g Zd_g  with  Zd_g = H[:, F_g] Vd[:, F_g]^T,  so what the
+ * ranks exchange is the narrow fp32 Zd[T, r_down] (r_down / d of the bytes of the paper's all-reduce of Y), and
+ * every rank finishes with the replicated Ud:
+ *   svdmlp_forward_partial  Zd_out[T, r_down] (fp32) = (SiLU((X Vg^T) Ug^T) .* ((X Vu^T) Uu^T)) Vd^T   of this handle
+ *   (the caller sums Zd_out over the shards: an all-reduce)
+ *   svdmlp_forward_finish   Y[T, d] = Zd Ud^T,  Zd fp32 [T, r_down] (rounded to fp16 as the product's operand for T > 32)
+ * Both are asynchronous on `stream`.  svdmlp_forward_partial followed by svdmlp_forward_finish on the same handle
+ * with nothing added in between equals svdmlp_forward.  For T <= 32 the pair runs on the register-streaming
+ * decode kernels (the one-kernel decode path cannot stop half way).  Errors as svdmlp_forward.
+ */
+int svdmlp_forward_partial(svdmlp_t* h, const void* X, int T, float* Zd_out, void* stream);
+int svdmlp_forward_finish(svdmlp_t* h, const float* Zd, int T, void* Y, void* stream);
+
+/*
  * The paper's XUV operator (Section 4.2.1):  Y[T, out] = (X[T, in] V^T) U^T  with U[out, r],
  * V[r, in]; X, U, V, Y bf16.  `workspace` is caller-owned device scratch of at least
  * svdlinear_workspace_bytes(T, in, out, r) bytes, 256-byte aligned; its contents are

@@ -26,6 +26,7 @@ FLAG_DECODE_COOPERATIVE = 0x400
 FLAG_TOKEN_SLABS = 0x800
 
 EXPORTS = ["svdmlp_create", "svdmlp_forward", "svdmlp_forward_host", "svdmlp_forward_prenorm_residual",
+           "svdmlp_forward_partial", "svdmlp_forward_finish",
            "svdlinear_forward", "svdlinear_workspace_bytes", "svdlinear_forward_noalloc",
            "svdlinear_create", "svdlinear_apply", "svdlinear_destroy", "svdmlp_destroy", "svdmlp_strerror",
            "svdmlp_last_device_status", "svdmlp_launch_count", "svdmlp_path_name",
@@ -53,6 +54,10 @@ def lib() -> ctypes.CDLL:
         L.svdmlp_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, ci, cu, vp]
         L.svdmlp_forward.restype = ci
         L.svdmlp_forward.argtypes = [vp, vp, ci, vp, vp]
+        L.svdmlp_forward_partial.restype = ci
+        L.svdmlp_forward_partial.argtypes = [vp, vp, ci, vp, vp]
+        L.svdmlp_forward_finish.restype = ci
+        L.svdmlp_forward_finish.argtypes = [vp, vp, ci, vp, vp]
         L.svdmlp_forward_host.restype = ci
         L.svdmlp_forward_host.argtypes = [vp, vp, ci, vp, vp]
         L.svdmlp_forward_prenorm_residual.restype = ci
@@ -160,6 +165,23 @@ def svdmlp_forward(h: Handle, X: torch.Tensor, Y: torch.Tensor | None = None, st
     if Y is None:
         Y = torch.empty((T, h.d), dtype=torch.float32 if h.flags & FLAG_Y_FP32 else torch.bfloat16, device=X.device)
     _check(lib().svdmlp_forward(h.ptr, _ptr(X), T, _ptr(Y), _stream(stream)), "svdmlp_forward")
+    return Y
+
+
+def svdmlp_forward_partial(h: Handle, X: torch.Tensor, Zd: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """This handle's (shard's) fp32 Zd[T, r_down]; the caller sums it over the shards."""
+    T = X.shape[0]
+    if Zd is None:
+        Zd = torch.empty((T, h._keep[4].shape[1]), dtype=torch.float32, device=X.device)
+    _check(lib().svdmlp_forward_partial(h.ptr, _ptr(X), T, _ptr(Zd), _stream(stream)), "svdmlp_forward_partial")
+    return Zd
+
+
+def svdmlp_forward_finish(h: Handle, Zd: torch.Tensor, Y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    T = Zd.shape[0]
+    if Y is None:
+        Y = torch.empty((T, h.d), dtype=torch.float32 if h.flags & FLAG_Y_FP32 else torch.bfloat16, device=Zd.device)
+    _check(lib().svdmlp_forward_finish(h.ptr, _ptr(Zd), T, _ptr(Y), _stream(stream)), "svdmlp_forward_finish")
     return Y
 
 

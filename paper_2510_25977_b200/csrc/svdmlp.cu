@@ -355,6 +355,7 @@ struct svdmlp {
     // cached X map and output maps of the TMA-store epilogues (box [32 rows, 64 columns])
     const void* x_ptr; int x_T; CUtensorMap mX;
     CUtensorMap mHc, mYc; const void* y_ptr; int y_T, y_f32;
+    float* zd_out32;                  // svdmlp_forward_partial: where the fp32 Zd of this call goes (else NULL)
     SlabPlan slabs;                   // token slabs of the gate/up -> down-1 pair for the last T seen (maps cached)
     CUtensorMap mUg64, mUu64, mUd64;  // half-tile boxes [64 rows, 64 columns] for the CTA-pair kernels
     CUtensorMap mVg64, mVu64, mVg128, mVu128, mVdHalf;  // half-tile boxes of the first-GEMM factors
@@ -594,7 +595,7 @@ int launch_convert(const void* in, __half* out, long n, int* flag, cudaStream_t 
     return SVDMLP_OK;
 }
 
-int launch_reduce(const float* part, int ksplit, long split_stride, long n, __half* out, cudaStream_t s) {
+int launch_reduce(const float* part, int ksplit, long split_stride, long n, __half* out, cudaStream_t s, float* out32 = nullptr) {
     int blocks = (int)std::min<long>((n / 4 + 255) / 256, 4 * num_sms());
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(std::max(blocks, 1)); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = s;
@@ -602,7 +603,7 @@ int launch_reduce(const float* part, int ksplit, long split_stride, long n, __ha
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, tensorpath::reduce_partials_kernel, part, ksplit, split_stride, n, out));
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, tensorpath::reduce_partials_kernel, part, ksplit, split_stride, n, out, out32));
     return SVDMLP_OK;
 }
 
@@ -643,7 +644,7 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     if (!h->tensor_ok) return SVDMLP_ERR_UNSUPPORTED;
     const int R = h->rg + h->ru;
     int rc;
-    if (h->x_ptr != X || h->x_T != T) {
+    if ((h->stage_mask & 1u) && (h->x_ptr != X || h->x_T != T)) {
         if ((rc = make_map(&h->mX, X, T, h->d, h->d, BM)) != SVDMLP_OK) return rc;
         h->x_ptr = X; h->x_T = T;
     }
@@ -732,7 +733,7 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     }
     }
     if (mask & 4u) {
-    { ProfScope ps(h, "down1_reduce", s); rc = launch_reduce(h->part, down1_ksplit, (long)T * h->rd, (long)T * h->rd, h->Zd16, s); }
+    { ProfScope ps(h, "down1_reduce", s); rc = launch_reduce(h->part, down1_ksplit, (long)T * h->rd, (long)T * h->rd, h->Zd16, s, h->zd_out32); }
     if (rc != SVDMLP_OK) return rc;
     h->launches += 1;
     }
@@ -1029,6 +1030,80 @@ int svdmlp_forward_prenorm_residual(svdmlp_t* h, const float* h_in, float* h_out
     CUDA_TRY(cudaGetLastError());
     h->launches += 1;
     return forward_impl(h, h->Xn, T, h_out, 1, h_in, s, true);
+}
+
+// ---- tensor-parallel halves of the forward pass ------------------------------------------------------------
+int svdmlp_forward_partial(svdmlp_t* h, const void* X, int T, float* Zd_out, void* stream) {
+    if (h == nullptr || X == nullptr || Zd_out == nullptr || T <= 0 || T > h->max_T) return SVDMLP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Zd_out)) return SVDMLP_ERR_ALIGNMENT;
+    if (h->stage_mask != ~0u) return SVDMLP_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const __nv_bfloat16* Xb = (const __nv_bfloat16*)X;
+    h->prof_n = 0;
+    if (use_skinny(h, T)) {
+        // register-streaming kernels: the first two of the three, which leave Zd in the handle's fp32 accumulator
+        if (T > h->t_skinny || h->Zs == nullptr) return SVDMLP_ERR_UNSUPPORTED;
+        int nt = T <= 8 ? 1 : T <= 16 ? 2 : 4;
+        while (nt > 1 && skinny_smem_need(h, nt) > 227 * 1024) nt >>= 1;
+        if (skinny_smem_need(h, nt) > 227 * 1024) return SVDMLP_ERR_UNSUPPORTED;
+        h->stage_mask = 1u | 2u;
+        const int rc = nt == 1 ? skinny_forward_nt<1>(h, Xb, T, nullptr, 0, nullptr, s)
+                     : nt == 2 ? skinny_forward_nt<2>(h, Xb, T, nullptr, 0, nullptr, s)
+                               : skinny_forward_nt<4>(h, Xb, T, nullptr, 0, nullptr, s);
+        h->stage_mask = ~0u;
+        if (rc != SVDMLP_OK) return rc;
+        CUDA_TRY(cudaMemcpyAsync(Zd_out, h->Zds, (size_t)T * h->rd * 4, cudaMemcpyDeviceToDevice, s));
+        // the third kernel, which is not run, would have cleared the first product's accumulator
+        CUDA_TRY(cudaMemsetAsync(h->Zs, 0, (size_t)h->t_skinny * (h->rg + h->ru) * 4, s));
+        return SVDMLP_OK;
+    }
+    h->stage_mask = 1u | 2u | 4u;
+    h->zd_out32 = Zd_out;
+    const int rc = tensor_forward(h, Xb, T, nullptr, 0, nullptr, s);
+    h->zd_out32 = nullptr;
+    h->stage_mask = ~0u;
+    return rc;
+}
+
+int svdmlp_forward_finish(svdmlp_t* h, const float* Zd, int T, void* Y, void* stream) {
+    if (h == nullptr || Zd == nullptr || Y == nullptr || T <= 0 || T > h->max_T) return SVDMLP_ERR_INVALID_ARG;
+    if (!aligned16(Zd) || !aligned16(Y)) return SVDMLP_ERR_ALIGNMENT;
+    if (h->stage_mask != ~0u) return SVDMLP_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int y_fp32 = (h->flags & SVDMLP_FLAG_Y_FP32) ? 1 : 0;
+    h->prof_n = 0;
+    if (use_skinny(h, T)) {
+        using namespace skinny;
+        int nt = T <= 8 ? 1 : T <= 16 ? 2 : 4;
+        while (nt > 1 && (size_t)nt * 8 * 2 * (h->rd + kPad) * 2 > 227 * 1024) nt >>= 1;
+        const size_t smem = (size_t)nt * 8 * 2 * (h->rd + kPad) * 2;
+        if (smem > 227 * 1024) return SVDMLP_ERR_UNSUPPORTED;
+        const int chunks = (T + nt * 8 - 1) / (nt * 8);
+        dim3 grid((h->d + 63) / 64, 1, chunks);
+#define SVDMLP_FINISH(NT)                                                                                              \
+        {                                                                                                              \
+            if (smem > 48 * 1024)                                                                                      \
+                CUDA_TRY(cudaFuncSetAttribute(expand_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)); \
+            expand_kernel<NT><<<grid, 128, smem, s>>>(Zd, T, h->rd, h->Ud, h->d, Y, y_fp32, nullptr, nullptr, 0);    \
+        }
+        if (nt == 1) SVDMLP_FINISH(1) else if (nt == 2) SVDMLP_FINISH(2) else SVDMLP_FINISH(4)
+#undef SVDMLP_FINISH
+        CUDA_TRY(cudaGetLastError());
+        h->launches += 1;
+        return SVDMLP_OK;
+    }
+    if (!h->tensor_ok) return SVDMLP_ERR_UNSUPPORTED;
+    {
+        const long n = (long)T * h->rd;
+        const int blocks = (int)std::min<long>((n / 4 + 255) / 256, 4 * num_sms());
+        tensorpath::f32_to_f16_kernel<<<std::max(blocks, 1), 256, 0, s>>>(Zd, h->Zd16, n);
+        CUDA_TRY(cudaGetLastError());
+        h->launches += 1;
+    }
+    h->stage_mask = 8u;
+    const int rc = tensor_forward(h, nullptr, T, Y, y_fp32, nullptr, s);
+    h->stage_mask = ~0u;
+    return rc;
 }
 
 int svdmlp_destroy(svdmlp_t* h) {

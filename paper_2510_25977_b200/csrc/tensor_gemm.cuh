@@ -922,9 +922,10 @@ bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ in, __half* __restrict__ ou
     if (bad) atomicExch(flag, 1);
 }
 
-// Sum split-K fp32 partials [ksplit][M, N] and write fp16 [M, N].
+// Sum split-K fp32 partials [ksplit][M, N] and write fp16 [M, N] (and, on request, the fp32 sums as well).
 __global__ void __launch_bounds__(256)
-reduce_partials_kernel(const float* __restrict__ part, int ksplit, long split_stride, long n, __half* __restrict__ out) {
+reduce_partials_kernel(const float* __restrict__ part, int ksplit, long split_stride, long n, __half* __restrict__ out,
+                       float* __restrict__ out32) {
     umma::pdl_launch_dependents();
     umma::pdl_wait();  // launched with programmatic stream serialization: the partials come from the previous grid
     for (long i = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < n; i += (long)gridDim.x * blockDim.x * 4) {
@@ -933,6 +934,21 @@ reduce_partials_kernel(const float* __restrict__ part, int ksplit, long split_st
             float4 v = *reinterpret_cast<const float4*>(part + k * split_stride + i);
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
         }
+        uint2 w;
+        w.x = pack_f16(s.x, s.y);
+        w.y = pack_f16(s.z, s.w);
+        *reinterpret_cast<uint2*>(out + i) = w;
+        if (out32 != nullptr) *reinterpret_cast<float4*>(out32 + i) = s;   // the unrounded sum, for a caller that adds shards
+    }
+}
+
+// fp32 [n] -> fp16 [n] (n a multiple of 4): a sum of partial Zd shards becomes the operand of the last product.
+__global__ void __launch_bounds__(256)
+f32_to_f16_kernel(const float* __restrict__ in, __half* __restrict__ out, long n) {
+    umma::pdl_launch_dependents();
+    umma::pdl_wait();
+    for (long i = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < n; i += (long)gridDim.x * blockDim.x * 4) {
+        const float4 s = *reinterpret_cast<const float4*>(in + i);
         uint2 w;
         w.x = pack_f16(s.x, s.y);
         w.y = pack_f16(s.z, s.w);
