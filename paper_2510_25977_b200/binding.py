@@ -24,6 +24,7 @@ FLAG_NO_TMEM_STRIP = 0x100
 FLAG_NO_WIDE_GATEUP = 0x200
 FLAG_DECODE_COOPERATIVE = 0x400
 FLAG_TOKEN_SLABS = 0x800
+FLAG_NO_FUSED_DOWN1 = 0x1000
 
 EXPORTS = ["svdmlp_create", "svdmlp_forward", "svdmlp_forward_host", "svdmlp_forward_prenorm_residual",
            "svdmlp_forward_partial", "svdmlp_forward_finish",

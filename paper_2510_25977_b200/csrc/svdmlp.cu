@@ -22,6 +22,7 @@
 #include "skinny.cuh"
 #include "tensor_gemm.cuh"
 #include "gateup_ts.cuh"
+#include "mlp_fused_ts.cuh"
 #include "gateup_wide.cuh"
 
 namespace {
@@ -249,6 +250,46 @@ int launch_gateup_ts(const GemmPlan& g, cudaStream_t s) {
     return SVDMLP_OK;
 }
 
+
+// Gate+up, SiLU and the first down product in one kernel with H kept on chip (mlp_fused_ts.cuh): ranks up to 128.
+int launch_gateup_down1_fused(const GemmPlan& g, cudaStream_t s) {
+    static bool attr_set = false;
+    static int attr_dev = -1;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set || attr_dev != dev) {
+        CUDA_TRY(cudaFuncSetAttribute(tensorpath::gateup_down1_ts_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      tensorpath::kFuSmemBytes));
+        attr_set = true;
+        attr_dev = dev;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(g.grid); cfg.blockDim = dim3(tensorpath::kPairThreads); cfg.dynamicSmemBytes = tensorpath::kFuSmemBytes; cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, tensorpath::gateup_down1_ts_pair_kernel, g.p));
+    return SVDMLP_OK;
+}
+
+// Segments per row-strip pair for the fused kernel: units = pairs x S should fill whole rounds of the CTA pairs.
+// Returns 0 if no S <= 16 keeps at least three quarters of the pairs busy (few tokens: the unfused kernels, which
+// split finer, are the better choice).
+int fused_segments(int T, int ffn, int rd, size_t part_elems) {
+    const int nc = std::max(1, num_sms() / 2), pairs_m = (T + 255) / 256, tiles_n = (ffn + 127) / 128;
+    double best = 0.0;
+    int best_s = 0;
+    for (int S = 1; S <= 16 && S <= tiles_n; ++S) {
+        if ((size_t)S * T * rd > part_elems) break;
+        const int units = pairs_m * S, rounds = (units + nc - 1) / nc;
+        const double eff = (double)units / ((double)rounds * nc);
+        if (eff > best + 0.03) { best = eff; best_s = S; }   // a finer split must buy 3 % to be worth shorter units
+    }
+    return best >= 0.75 ? best_s : 0;
+}
 
 // Tile width of Zd = H Vd^T (N = r_down): 256 unless the padding of N to whole tiles wastes much more than with
 // 128-wide tiles (r = 320: 512 against 384 columns).
@@ -683,6 +724,25 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     const SlabPlan* sp = slab_plan(h, T);
     if (sp == nullptr) return SVDMLP_ERR_CUDA;
     int down1_ksplit = 0;
+    // Ranks up to 128: both products in one kernel, H stays in shared memory (mlp_fused_ts.cuh)
+    const int fused_S = ((mask & 6u) == 6u && sp->n == 1 && pairs_ok && h->rg == h->ru && h->rg <= 128 && h->rd <= 128 &&
+                         !(h->flags & (SVDMLP_FLAG_NO_TMEM_STRIP | SVDMLP_FLAG_NO_FUSED_DOWN1)))
+                            ? fused_segments(T, h->ffn, h->rd, h->part_elems) : 0;
+    if (fused_S > 0) {
+        plan_gemm(g, 2, 128, true, false, T, h->ffn, h->rg, 1, true, true);
+        g.p.tmA[0] = h->mZg; g.p.tmA[1] = h->mZu;
+        g.p.tmB[0] = h->mUg64; g.p.tmB[1] = h->mUu64;
+        g.p.tmC = h->mVdHalf;
+        g.p.a_fmt = umma::kFmtF16; g.p.b_fmt = umma::kFmtF16; g.p.status = h->status_dev;
+        g.p.C = h->part; g.p.ldc = h->rd; g.p.split_stride = (long)T * h->rd; g.p.out_mode = OUT_F32;
+        g.p.ksplit = fused_S; g.p.stages = tensorpath::kFuSlots;
+        g.grid = 2 * std::min(((g.p.tiles_m + 1) / 2) * fused_S, num_sms() / 2);
+        { ProfScope ps(h, "gateup_down1", s); rc = launch_gateup_down1_fused(g, s); }
+        if (rc != SVDMLP_OK) return rc;
+        { ProfScope ps(h, "down1_reduce", s); rc = launch_reduce(h->part, fused_S, (long)T * h->rd, (long)T * h->rd, h->Zd16, s, h->zd_out32); }
+        if (rc != SVDMLP_OK) return rc;
+        h->launches += 2;
+    } else {
     for (int si = 0; si < sp->n; ++si) {
     const int row0 = si * sp->rows, Ts = std::min(sp->rows, T - row0);
     const SlabMaps& sm = sp->maps[si];
@@ -737,6 +797,7 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     if (rc != SVDMLP_OK) return rc;
     h->launches += 1;
     }
+    }   // not fused
     // 4. Y = Zd Ud^T   (phase 2 of the XUV chain)
     if (mask & 8u) {
     const bool y_tma = true;  // bf16 and fp32 (+ residual) outputs both leave through TMA stores

@@ -390,3 +390,33 @@ def test_svdlinear_handle_reports_factors_outside_the_fp16_range():
     torch.cuda.synchronize()
     assert torch.isfinite(Y.float()).all()
     binding.svdlinear_destroy(h)
+
+
+@pytest.mark.parametrize("r,rd,T", [(72, 40, 1100), (64, 128, 1500), (128, 128, 1030), (32, 64, 2600)])
+def test_fused_gateup_down1_ragged(oracle, r, rd, T):
+    """Ranks up to 128: gate/up, SiLU and the first down product as one kernel with H kept in shared memory, on
+    ragged shapes (partial last row strip, ffn tile and K chunk; one and two K chunks; several units per CTA pair),
+    against the oracle and against the same handle shape with the fused kernel switched off."""
+    d, ffn = 512, 2200
+    f = inputs.direct_factors(d, ffn, r, seed=21, r_down=rd, device="cuda")
+    X = inputs.activations(T, d, seed=21, device="cuda")
+    rows = inputs.rows_of_every_tile(T, per_tile=3)
+    ref = _gpu.oracle_rows(oracle, f, X, rows)
+    Y = _gpu.run_mlp(f, X, flags=TENSOR)
+    _gpu.assert_close(Y[rows], ref, f"fused r={r} rd={rd} T={T}")
+    Y2 = _gpu.run_mlp(f, X, flags=TENSOR | binding.FLAG_NO_FUSED_DOWN1)
+    _gpu.assert_close(Y2[rows], ref, f"unfused r={r} rd={rd} T={T}")
+
+
+def test_fused_gateup_down1_repeated_launches(oracle):
+    """Back-to-back forwards on one handle (ring phases, H buffers and the Zd accumulator carry over units, not launches)."""
+    f = inputs.direct_factors(1024, 4096, 128, seed=22, device="cuda")
+    h = binding.svdmlp_create(*f.tensors(), max_T=2048)
+    for i, T in enumerate((2048, 1024, 2048)):
+        X = inputs.activations(T, 1024, seed=30 + i, device="cuda")
+        Y = binding.svdmlp_forward(h, X)
+        torch.cuda.synchronize()
+        assert binding.svdmlp_last_device_status(h) == 0
+        rows = inputs.rows_of_every_tile(T, per_tile=2)
+        _gpu.assert_close(Y[rows], _gpu.oracle_rows(oracle, f, X, rows), f"fused repeat {i}")
+    binding.svdmlp_destroy(h)
