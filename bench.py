@@ -216,7 +216,7 @@ def time_steps(rep, steps, warmup, dist_ctx=None, use_graph=True):
     return ms, launches
 
 
-STAGE_BITS = {"stage1": 1, "gateup": 2, "down1": 4, "down2": 8, "rmsnorm": 16}
+STAGE_BITS = {"stage1": 1, "gateup": 2, "down1": 4, "down2": 8, "rmsnorm": 16, "gateup_down1": 6}
 
 
 def kernel_breakdown(rep, steps):
@@ -230,8 +230,9 @@ def kernel_breakdown(rep, steps):
     b = rep.binding
     handles = [h for hs in rep.handles for h in hs]
     out = {}
-    if rep.path() == "tensor":
-        names = ["stage1", "gateup", "down1", "down2"] + (["rmsnorm"] if rep.stack else [])
+    if rep.path().startswith("tensor"):
+        mid = ["gateup_down1"] if rep.path() == "tensor-fused" else ["gateup", "down1"]
+        names = ["stage1"] + mid + ["down2"] + (["rmsnorm"] if rep.stack else [])
         for name in names:
             for h in handles:
                 b.svdmlp_stage_mask(h, STAGE_BITS[name])
@@ -273,6 +274,7 @@ def kernel_algorithmic_work(name, T, d, ffn, r, layers, path):
             "gateup": (2 * 2 * ffn * r + 2 * T * 2 * r + 2 * T * ffn, 4 * T * ffn * r),
             "down1": (2 * r * ffn + 2 * T * ffn + 4 * T * r, 2 * T * ffn * r),
             "down2": (2 * d * r + 2 * T * r + 2 * T * d, 2 * T * r * d),
+            "gateup_down1": (2 * 3 * ffn * r + 2 * T * 2 * r + 4 * T * r, 6 * T * ffn * r),
             "rmsnorm": (6 * T * d, 3 * T * d),
             "stage1_reduce": (0, 0), "down1_reduce": (0, 0),
         }
@@ -608,7 +610,7 @@ def main():
             "config": {"workload": args.workload, "d": CFG[cfg]["d"], "ffn": CFG[cfg]["ffn"], "r": r, "T": T_global,
                        "layers": CFG[cfg]["layers"], "path": point["path"],
                        "parallelism": (f"token rows of one {world * T_global}-row batch sharded x{world}, no collective"
-                                       if point["path"] == "tensor" else f"replicas x{world}"),
+                                       if point["path"].startswith("tensor") else f"replicas x{world}"),
                        "l2_policy": f"inputs larger than L2: {point['replicas']} rotating replicas of factors and activations",
                        "timed_region": "one CUDA graph of all timed steps, CUDA events on the launching stream"},
             "tflops": point["tflops"] * world, "alg_gbs": point["alg_gbs"] * world,

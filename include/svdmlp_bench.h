@@ -48,7 +48,8 @@ const char* svdmlp_profile_name(const svdmlp_t* h, int index);
  */
 int svdmlp_stage_mask(svdmlp_t* h, unsigned mask);
 
-/* Name of the kernel path the handle would use for T tokens: "skinny" or "tensor". */
+/* Name of the kernel path the handle would use for T tokens: "skinny", "tensor", or "tensor-fused" (large T with
+ * gate/up and the first down product in one kernel: ranks up to 128). */
 const char* svdmlp_path_name(const svdmlp_t* h, int T);
 
 #ifdef __cplusplus

@@ -17,28 +17,36 @@
 // CTA pair (cta_group::2) as in gateup_ts.cuh: each CTA owns 128 token rows and loads 64 rows of every factor tile.
 // Ring slots (16 KiB): a [128 x 64] strip chunk, or two [64 x 64] chunks of Ug / Uu / Vd; a tile takes three slots
 // (G, Up, Vd) and the ring has a multiple of three, so inside a unit a slot always serves the same consumer.
-// Warps: 0 and 11 TMA producers (alternate slots); 1 issues G and copies the strips; 10 issues Up and, one tile
-// behind, the Zd MMAs; 2-9 epilogue (lane quadrant x column half).  Every wait is bounded.
+// Warps: 0 and 11 TMA producers (alternate slots); 1 issues G and copies the strips, 10 issues Up, 12 issues the Zd
+// MMAs (one thread issues a tcgen05.mma about every 55 cycles: two issuers for the 24 MMAs of a tile were the
+// kernel's bound); 2-9 epilogue (lane quadrant x column half).  Ring slots change hands between the issuers only
+// at unit boundaries, where `adone` / `aready` order every earlier fill before the first wait that follows
+// (one-bit phase parities cannot tell a fill that has not landed from the one two fills later).  Every wait is bounded.
 #pragma once
 #include "gateup_ts.cuh"
 
 namespace tensorpath {
 
-constexpr int kFuSlots = 9;
+constexpr int kFuSlots = 12;
+constexpr int kFuHBufs = 1;                                 // H tiles in shared memory (one: its Zd MMAs end long before the epilogue has the next tile)
+constexpr int kFuThreads = 13 * 32;                          // the pair kernels' twelve warps + warp 12, the Zd issuer
+constexpr int kFuZdWarp = 12;
 constexpr int kFuHBytes = kEpiWarps * 4096;                 // one [128 x 128] fp16 tile of H per CTA
 constexpr int kFuBarrierBytes = (2 * kFuSlots + 16) * 8 + 16;
-constexpr int kFuSmemBytes = 1024 + kFuSlots * kTsSlotBytes + 2 * kFuHBytes + kFuBarrierBytes;
+constexpr int kFuSmemBytes = 1024 + kFuSlots * kTsSlotBytes + kFuHBufs * kFuHBytes + kFuBarrierBytes;
+static_assert(kFuSlots % 3 == 0, "inside a unit a ring slot must always serve the same issuer");
+static_assert(kFuSmemBytes <= 232448, "shared memory of one SM");
 
 // p: tmA[0/1] = Zg / Zu ([T, r] fp16, box [128, 64]); tmB[0/1] = Ug / Uu ([ffn, r] fp16, box [64, 64]);
 // tmC = Vd ([r_down, ffn] fp16, box [64, 64]); C = fp32 partials [ksplit][T, ldc], ldc = r_down,
 // split_stride = T r_down; M = T, N = ffn, K = r <= 128; tiles_m = ceil(T / 128), tiles_n = ceil(ffn / 128),
 // chunks_total = ceil(r / 64); ksplit = S segments per row-strip pair (S <= tiles_n); stages = kFuSlots.
-__global__ void __launch_bounds__(kPairThreads, 1) gateup_down1_ts_pair_kernel(const __grid_constant__ GemmParams p) {
+__global__ void __launch_bounds__(kFuThreads, 1) gateup_down1_ts_pair_kernel(const __grid_constant__ GemmParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (umma::smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* ring = smem;
-    unsigned char* hbuf = ring + kFuSlots * kTsSlotBytes;    // two H tiles, 1024-byte aligned
-    uint64_t* full = reinterpret_cast<uint64_t*>(hbuf + 2 * kFuHBytes);
+    unsigned char* hbuf = ring + kFuSlots * kTsSlotBytes;    // the H tile(s), 1024-byte aligned
+    uint64_t* full = reinterpret_cast<uint64_t*>(hbuf + kFuHBufs * kFuHBytes);
     uint64_t* empty = full + kFuSlots;
     uint64_t* tfull = empty + kFuSlots;   // [branch]
     uint64_t* tempty = tfull + 2;         // [branch]
@@ -70,7 +78,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_down1_ts_pair_kernel(c
             umma::mbar_init(&tfull[a], 1); umma::mbar_init(&tempty[a], 2 * kEpiWarps);
             umma::mbar_init(&hready[a], 2 * kEpiWarps); umma::mbar_init(&hfree[a], 1);
         }
-        umma::mbar_init(adone, 2);
+        umma::mbar_init(adone, 3);   // one commit per issuer warp at the end of a unit
         umma::mbar_init(aready, 1);
         umma::mbar_init(zfull, 1);
         umma::mbar_init(zempty, 2 * kEpiWarps);
@@ -210,41 +218,13 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_down1_ts_pair_kernel(c
             }
         }
     } else if (warp == 10) {
-        if (leader) {  // ---------------- tcgen05 issuer of Up and, one tile behind, of Zd += H Vd^T ----------------
+        if (leader) {  // ---------------- tcgen05 issuer of Up ----------------
             const uint32_t idesc = umma::make_idesc(p.a_fmt, p.b_fmt, 2 * BM, 128);
             int stage = 0;
             uint32_t phase = 0, ph = 0, strip_phase = 0;
-            int g = 0;            // tiles handled so far by this CTA pair: H buffer g & 1, its phase (g >> 1) & 1
-            int ui = 0;           // units handled so far
             bool ok = true;
             auto skip_slots = [&](int k) { stage += k; while (stage >= nslot) { stage -= nslot; phase ^= 1; } };
-            // Zd += H(tile) Vd(tile)^T from H buffer hb and the Vd slot (vstage, vphase); `first`: first tile of the unit
-            auto issue_zd = [&](int hb, uint32_t hphase, int vstage, uint32_t vphase, bool first, bool last) -> bool {
-                if (!umma::mbar_wait_warp(&hready[hb], hphase, abort_flag)) return false;
-                if (!umma::mbar_wait_warp(&full[vstage], vphase, abort_flag)) return false;
-                // the accumulator of the previous unit has been read out before the first MMA overwrites it
-                if (first && !umma::mbar_wait_warp(zempty, (uint32_t)(ui & 1) ^ 1u, abort_flag)) return false;
-                umma::tc_fence_after_sync();
-                if (umma::elect_one()) {
-                    const uint32_t ha = umma::smem_u32(hbuf + hb * kFuHBytes), va = umma::smem_u32(ring + vstage * kTsSlotBytes);
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const uint64_t ad = umma::smem_desc_sw128(ha + j * (kFuHBytes / 2)), bd = umma::smem_desc_sw128(va + j * kTsChunkBytes);
-#pragma unroll
-                        for (int kk = 0; kk < BK / 16; ++kk)
-                            umma::mma_f16_ss_pair(tmem_base + 128, ad + 2 * kk, bd + 2 * kk, idesc, !first || j > 0 || kk > 0);
-                    }
-                    umma::mma_commit_pair(&empty[vstage]);
-                    umma::mma_commit_pair(&hfree[hb]);
-                    // `adone` here, not after the unit's last Up: this warp's ring slots of the unit (Up, Vd) have then
-                    // all been consumed, so the other issuer may wait on slots whose previous fill was this warp's
-                    // (one-bit phase parities cannot tell a fill that has not landed from the one two fills later)
-                    if (last) { umma::mma_commit_pair(zfull); umma::mma_commit_pair(adone); }
-                }
-                __syncwarp();
-                return true;
-            };
-            for (int u = cluster_id; u < units && ok; u += nclusters, ++ui) {
+            for (int u = cluster_id; u < units && ok; u += nclusters) {
                 int mp, seg, n0, n1;
                 unit_tiles(u, mp, seg, n0, n1);
                 skip_slots(2 * chunks);
@@ -252,8 +232,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_down1_ts_pair_kernel(c
                 if (!ok) break;
                 umma::tc_fence_after_sync();
                 strip_phase ^= 1;
-                int pv_stage = -1; uint32_t pv_phase = 0;   // Vd slot of the previous tile of this unit
-                for (int n = n0; n < n1 && ok; ++n, ++g) {
+                for (int n = n0; n < n1 && ok; ++n) {
                     skip_slots(spb);  // G's slots of this tile
                     ok = umma::mbar_wait_warp(&tempty[1], ph ^ 1, abort_flag);
                     if (!ok) break;
@@ -276,16 +255,58 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_down1_ts_pair_kernel(c
                         if (++stage == nslot) { stage = 0; phase ^= 1; }
                     }
                     if (!ok) break;
-                    if (umma::elect_one()) umma::mma_commit_pair(&tfull[1]);
+                    if (umma::elect_one()) {
+                        umma::mma_commit_pair(&tfull[1]);
+                        if (n + 1 == n1) umma::mma_commit_pair(adone);
+                    }
                     __syncwarp();
                     ph ^= 1;
-                    const int vstage = stage; const uint32_t vphase = phase;   // this tile's Vd slot
-                    skip_slots(1);
-                    if (pv_stage >= 0)   // the previous tile's H has been built while this tile's G and Up ran
-                        ok = issue_zd((g - 1) & 1, (uint32_t)((g - 1) >> 1) & 1u, pv_stage, pv_phase, n - 1 == n0, false);
-                    pv_stage = vstage; pv_phase = vphase;
+                    skip_slots(1);  // Vd's slot of this tile
                 }
-                if (ok && pv_stage >= 0) ok = issue_zd((g - 1) & 1, (uint32_t)((g - 1) >> 1) & 1u, pv_stage, pv_phase, n1 - 1 == n0, true);
+            }
+        }
+    } else if (warp == kFuZdWarp) {
+        if (leader) {  // ---------------- tcgen05 issuer of Zd += H Vd^T (a tile behind the other two by construction) ----------------
+            const uint32_t idesc = umma::make_idesc(p.a_fmt, p.b_fmt, 2 * BM, 128);
+            int stage = 0;
+            uint32_t phase = 0, strip_phase = 0;
+            int g = 0;            // tiles handled so far by this CTA pair: H buffer g % kFuHBufs, its phase (g / kFuHBufs) & 1
+            int ui = 0;           // units handled so far
+            bool ok = true;
+            auto skip_slots = [&](int k) { stage += k; while (stage >= nslot) { stage -= nslot; phase ^= 1; } };
+            for (int u = cluster_id; u < units && ok; u += nclusters, ++ui) {
+                int mp, seg, n0, n1;
+                unit_tiles(u, mp, seg, n0, n1);
+                skip_slots(2 * chunks);
+                // every issuer has finished the previous unit (its ring slots are consumed): see `adone`
+                ok = umma::mbar_wait_warp(aready, strip_phase, abort_flag);
+                if (!ok) break;
+                strip_phase ^= 1;
+                for (int n = n0; n < n1 && ok; ++n, ++g) {
+                    skip_slots(2 * spb);  // G's and Up's slots of this tile
+                    const int hb = g % kFuHBufs;
+                    ok = umma::mbar_wait_warp(&hready[hb], (uint32_t)(g / kFuHBufs) & 1u, abort_flag) &&
+                         umma::mbar_wait_warp(&full[stage], phase, abort_flag);
+                    // the accumulator of the previous unit has been read out before the first MMA overwrites it
+                    if (ok && n == n0) ok = umma::mbar_wait_warp(zempty, (uint32_t)(ui & 1) ^ 1u, abort_flag);
+                    if (!ok) break;
+                    umma::tc_fence_after_sync();
+                    if (umma::elect_one()) {
+                        const uint32_t ha = umma::smem_u32(hbuf + hb * kFuHBytes), va = umma::smem_u32(ring + stage * kTsSlotBytes);
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            const uint64_t ad = umma::smem_desc_sw128(ha + j * (kFuHBytes / 2)), bd = umma::smem_desc_sw128(va + j * kTsChunkBytes);
+#pragma unroll
+                            for (int kk = 0; kk < BK / 16; ++kk)
+                                umma::mma_f16_ss_pair(tmem_base + 128, ad + 2 * kk, bd + 2 * kk, idesc, n > n0 || j > 0 || kk > 0);
+                        }
+                        umma::mma_commit_pair(&empty[stage]);
+                        umma::mma_commit_pair(&hfree[hb]);
+                        if (n + 1 == n1) { umma::mma_commit_pair(zfull); umma::mma_commit_pair(adone); }
+                    }
+                    __syncwarp();
+                    if (++stage == nslot) { stage = 0; phase ^= 1; }
+                }
             }
         }
     } else if (warp < 2 + kEpiWarps) {  // ---------------- epilogue warps 2..9 (both CTAs, own 128 rows) ----------------
@@ -346,10 +367,9 @@ __global__ void __launch_bounds__(kPairThreads, 1) gateup_down1_ts_pair_kernel(c
                         const __half2 r2 = __hmul2(*reinterpret_cast<const __half2*>(&sg[hh * 16 + j]), u2);
                         sg[hh * 16 + j] = *reinterpret_cast<const uint32_t*>(&r2);
                     }
-                // H tile into shared memory as the A operand of Zd += H Vd^T; the buffer's previous tile (two tiles
-                // back) has been multiplied
-                const int hb = g & 1;
-                ok = umma::mbar_wait_warp(&hfree[hb], ((uint32_t)(g >> 1) & 1u) ^ 1u, abort_flag);
+                // H tile into shared memory as the A operand of Zd += H Vd^T; the buffer's previous tile has been multiplied
+                const int hb = g % kFuHBufs;
+                ok = umma::mbar_wait_warp(&hfree[hb], ((uint32_t)(g / kFuHBufs) & 1u) ^ 1u, abort_flag);
                 if (!ok) break;
                 unsigned char* dst = hbuf + hb * kFuHBytes + my_off;
 #pragma unroll

@@ -264,7 +264,7 @@ int launch_gateup_down1_fused(const GemmPlan& g, cudaStream_t s) {
         attr_dev = dev;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(g.grid); cfg.blockDim = dim3(tensorpath::kPairThreads); cfg.dynamicSmemBytes = tensorpath::kFuSmemBytes; cfg.stream = s;
+    cfg.gridDim = dim3(g.grid); cfg.blockDim = dim3(tensorpath::kFuThreads); cfg.dynamicSmemBytes = tensorpath::kFuSmemBytes; cfg.stream = s;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
@@ -680,6 +680,14 @@ const SlabPlan* slab_plan(svdmlp* h, int T) {
     return &sp;
 }
 
+// Segments of the fused gate/up + down-1 kernel for this handle and T, 0 if the two-kernel form runs instead.
+int fused_plan(const svdmlp* h, int T) {
+    if (!h->tensor_ok || (h->flags & (SVDMLP_FLAG_NO_CTA_PAIRS | SVDMLP_FLAG_NO_TMEM_STRIP | SVDMLP_FLAG_NO_FUSED_DOWN1 | SVDMLP_FLAG_TOKEN_SLABS)))
+        return 0;
+    if (h->rg != h->ru || h->rg > 128 || h->rd > 128) return 0;
+    return fused_segments(T, h->ffn, h->rd, h->part_elems);
+}
+
 int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32, const float* resid, cudaStream_t s) {
     using namespace tensorpath;
     if (!h->tensor_ok) return SVDMLP_ERR_UNSUPPORTED;
@@ -725,9 +733,7 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     if (sp == nullptr) return SVDMLP_ERR_CUDA;
     int down1_ksplit = 0;
     // Ranks up to 128: both products in one kernel, H stays in shared memory (mlp_fused_ts.cuh)
-    const int fused_S = ((mask & 6u) == 6u && sp->n == 1 && pairs_ok && h->rg == h->ru && h->rg <= 128 && h->rd <= 128 &&
-                         !(h->flags & (SVDMLP_FLAG_NO_TMEM_STRIP | SVDMLP_FLAG_NO_FUSED_DOWN1)))
-                            ? fused_segments(T, h->ffn, h->rd, h->part_elems) : 0;
+    const int fused_S = ((mask & 6u) == 6u && sp->n == 1) ? fused_plan(h, T) : 0;
     if (fused_S > 0) {
         plan_gemm(g, 2, 128, true, false, T, h->ffn, h->rg, 1, true, true);
         g.p.tmA[0] = h->mZg; g.p.tmA[1] = h->mZu;
@@ -1251,7 +1257,8 @@ unsigned long long svdmlp_launch_count(const svdmlp_t* h) { return h ? h->launch
 
 const char* svdmlp_path_name(const svdmlp_t* h, int T) {
     if (h == nullptr) return "none";
-    return use_skinny(h, T) ? "skinny" : "tensor";
+    if (use_skinny(h, T)) return "skinny";
+    return fused_plan(h, T) > 0 ? "tensor-fused" : "tensor";
 }
 
 }  // extern "C"
