@@ -183,6 +183,25 @@ int svdlinear_forward_noalloc(const void* X, int T, int in, int out, int r, cons
  */
 int svdmlp_block_aligned_rank(int k, int n, double ratio, int block, double alpha);
 
+/*
+ * Compression front-end on the device (Section 4.1 with S = I, i.e. without the activation-aware whitening, which
+ * needs calibration data: Eq. 3 is then the plain SVD W = U Sigma V^T; Eq. 6-8 fold Sigma into the factors).
+ * W[out, in] is a dense fp32 weight on the device; the call writes the factors of the r largest singular values,
+ *     U_out[out, r] = U_r diag(sigma_r),  V_out[r, in] = V_r^T                    (flags = 0; W ~= U_out V_out), or
+ *     U_out = U_r diag(sqrt(sigma_r)),    V_out = diag(sqrt(sigma_r)) V_r^T        (SVDMLP_COMPRESS_SPLIT_SQRT: Eq. 6-7)
+ * as bf16 (round to nearest even), ready for svdmlp_create / svdlinear_create.  sigma_out, if not NULL, is a HOST
+ * array of min(out, in) floats that receives all singular values in descending order.  r = the value of
+ * svdmlp_block_aligned_rank (Eq. 5) or any 1 <= r <= min(out, in).  One-sided Jacobi in fp32 with fp64 dot
+ * products: singular values to about 1e-6 relative.  `workspace`: device scratch of at least
+ * svdmlp_compress_workspace_bytes(out, in) bytes, 256-byte aligned.  An offline step: the call synchronises
+ * `stream` several times (once per sweep) and returns when the factors are written.
+ * Errors: INVALID_ARG, ALIGNMENT, NOMEM (workspace too small), ARCH, CUDA.
+ */
+#define SVDMLP_COMPRESS_SPLIT_SQRT 0x1u
+int svdmlp_compress(const float* W, int out, int in, int r, void* U_out, void* V_out, float* sigma_out,
+                    void* workspace, size_t workspace_bytes, unsigned flags, void* stream);
+size_t svdmlp_compress_workspace_bytes(int out, int in);
+
 /* Free the workspace.  Waits for the device to finish work that uses it.  NULL is allowed. */
 int svdmlp_destroy(svdmlp_t* h);
 

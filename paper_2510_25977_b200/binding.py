@@ -29,7 +29,8 @@ FLAG_NO_FUSED_DOWN1 = 0x1000
 EXPORTS = ["svdmlp_create", "svdmlp_forward", "svdmlp_forward_host", "svdmlp_forward_prenorm_residual",
            "svdmlp_forward_partial", "svdmlp_forward_finish",
            "svdlinear_forward", "svdlinear_workspace_bytes", "svdlinear_forward_noalloc",
-           "svdlinear_create", "svdlinear_apply", "svdlinear_destroy", "svdmlp_destroy", "svdmlp_strerror",
+           "svdlinear_create", "svdlinear_apply", "svdlinear_destroy",
+           "svdmlp_compress", "svdmlp_compress_workspace_bytes", "svdmlp_destroy", "svdmlp_strerror",
            "svdmlp_last_device_status", "svdmlp_launch_count", "svdmlp_path_name",
            "svdmlp_profile_enable", "svdmlp_profile_read", "svdmlp_profile_name", "svdmlp_stage_mask",
            "svdmlp_block_aligned_rank", "svdmlp_selftest_timeout"]
@@ -67,6 +68,10 @@ def lib() -> ctypes.CDLL:
         L.svdlinear_forward.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.svdlinear_forward_noalloc.restype = ci
         L.svdlinear_forward_noalloc.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp]
+        L.svdmlp_compress.restype = ci
+        L.svdmlp_compress.argtypes = [vp, ci, ci, ci, vp, vp, ctypes.POINTER(ctypes.c_float), vp, ctypes.c_size_t, cu, vp]
+        L.svdmlp_compress_workspace_bytes.restype = ctypes.c_size_t
+        L.svdmlp_compress_workspace_bytes.argtypes = [ci, ci]
         L.svdlinear_create.restype = ci
         L.svdlinear_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, vp, vp, ci, vp]
         L.svdlinear_apply.restype = ci
@@ -260,6 +265,24 @@ def svdlinear_apply(h: LinearHandle, X, Y=None, stream=None) -> torch.Tensor:
 
 def svdlinear_destroy(h: LinearHandle):
     h.close()
+
+
+COMPRESS_SPLIT_SQRT = 0x1
+
+
+def svdmlp_compress(W: torch.Tensor, r: int, flags: int = 0, stream=None):
+    """Rank-r factors of a dense fp32 CUDA weight W[out, in]: (U[out, r], V[r, in]) bf16 and all singular values
+    (a CPU float tensor, descending)."""
+    if not (W.is_cuda and W.dtype == torch.float32 and W.is_contiguous()):
+        raise ValueError("W must be a contiguous fp32 CUDA tensor")
+    n_out, n_in = W.shape
+    U = torch.empty((n_out, r), dtype=torch.bfloat16, device=W.device)
+    V = torch.empty((r, n_in), dtype=torch.bfloat16, device=W.device)
+    sigma = (ctypes.c_float * min(n_out, n_in))()
+    ws = torch.empty(int(lib().svdmlp_compress_workspace_bytes(n_out, n_in)), dtype=torch.uint8, device=W.device)
+    _check(lib().svdmlp_compress(_ptr(W), n_out, n_in, r, _ptr(U), _ptr(V), sigma, _ptr(ws), ws.numel(), flags, _stream(stream)),
+           "svdmlp_compress")
+    return U, V, torch.tensor(list(sigma), dtype=torch.float32)
 
 
 NOALLOC_MAX_T = 32

@@ -16,6 +16,8 @@
 #include <string.h>
 
 #include <algorithm>
+#include <numeric>
+#include <vector>
 #include <new>
 
 #include "decode_persistent.cuh"
@@ -24,6 +26,7 @@
 #include "gateup_ts.cuh"
 #include "mlp_fused_ts.cuh"
 #include "gateup_wide.cuh"
+#include "compress.cuh"
 
 namespace {
 
@@ -1505,3 +1508,62 @@ int svdlinear_destroy(svdlinear_t* h) {
 
 }  // extern "C"
 
+// ---- compression front-end ---------------------------------------------------------------------------
+extern "C" size_t svdmlp_compress_workspace_bytes(int out, int in) {
+    if (out <= 0 || in <= 0) return 0;
+    const size_t n = (size_t)std::min(out, in), m = (size_t)std::max(out, in);
+    return ((n * m + n * n + n) * sizeof(float) + n * sizeof(int) + 256 + 255) & ~(size_t)255;
+}
+
+extern "C" int svdmlp_compress(const float* W, int out, int in, int r, void* U_out, void* V_out, float* sigma_out,
+                               void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
+    if (!W || !U_out || !V_out || !workspace || out <= 0 || in <= 0 || r <= 0 || r > std::min(out, in)) return SVDMLP_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return SVDMLP_ERR_ALIGNMENT;
+    if (workspace_bytes < svdmlp_compress_workspace_bytes(out, in)) return SVDMLP_ERR_NOMEM;
+    int rc = check_arch();
+    if (rc != SVDMLP_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int transpose = in <= out ? 1 : 0;           // the vectors made orthogonal: columns of W, or its rows
+    const int n = std::min(out, in), m = std::max(out, in), n_even = (n + 1) & ~1;
+    float* B = reinterpret_cast<float*>(workspace);
+    float* R = B + (size_t)n * m;
+    float* sigma = R + (size_t)n * n;
+    int* order = reinterpret_cast<int*>(sigma + n);
+    int* rotated = order + n;
+    const int blocks = std::min(8 * num_sms(), (int)std::min<size_t>(((size_t)n * m + 255) / 256, 1u << 20));
+    compress::init_kernel<<<std::max(blocks, 1), compress::kThreads, 0, s>>>(W, out, in, transpose, n, m, B, R);
+    CUDA_TRY(cudaGetLastError());
+    const int max_sweeps = 40;
+    const double tol = 1e-7;   // fp32 storage: pairs whose cosine is below this count as orthogonal
+    if (n > 1) {
+        for (int sweep = 0; sweep < max_sweeps; ++sweep) {
+            CUDA_TRY(cudaMemsetAsync(rotated, 0, sizeof(int), s));
+            for (int k = 0; k < n_even - 1; ++k)
+                compress::step_kernel<<<n_even / 2, compress::kThreads, 0, s>>>(B, R, n, m, n_even, k, tol, rotated);
+            CUDA_TRY(cudaGetLastError());
+            int h_rot = 0;
+            CUDA_TRY(cudaMemcpyAsync(&h_rot, rotated, sizeof(int), cudaMemcpyDeviceToHost, s));
+            CUDA_TRY(cudaStreamSynchronize(s));
+            if (h_rot == 0) break;
+        }
+    }
+    compress::norms_kernel<<<n, compress::kThreads, 0, s>>>(B, n, m, sigma);
+    CUDA_TRY(cudaGetLastError());
+    std::vector<float> hs(n);
+    CUDA_TRY(cudaMemcpyAsync(hs.data(), sigma, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+    std::vector<int> ho(n);
+    std::iota(ho.begin(), ho.end(), 0);
+    std::stable_sort(ho.begin(), ho.end(), [&](int a, int b) { return hs[a] > hs[b]; });
+    CUDA_TRY(cudaMemcpyAsync(order, ho.data(), (size_t)n * sizeof(int), cudaMemcpyHostToDevice, s));
+    if (sigma_out != nullptr)
+        for (int k = 0; k < n; ++k) sigma_out[k] = hs[ho[k]];   // HOST array, descending
+    const long total = (long)out * r + (long)r * in;
+    const int eb = (int)std::min<long>((total + 255) / 256, 8L * num_sms());
+    compress::emit_kernel<<<std::max(eb, 1), compress::kThreads, 0, s>>>(B, R, sigma, order, out, in, r, transpose, n, m,
+                                                                        (flags & SVDMLP_COMPRESS_SPLIT_SQRT) ? 1 : 0,
+                                                                        (__nv_bfloat16*)U_out, (__nv_bfloat16*)V_out);
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(s));   // `ho` is read by the copy above
+    return SVDMLP_OK;
+}
