@@ -279,18 +279,23 @@ int launch_gateup_down1_fused(const GemmPlan& g, cudaStream_t s) {
 }
 
 // Segments per row-strip pair for the fused kernel: units = pairs x S should fill whole rounds of the CTA pairs.
-// Returns 0 if no S <= 16 keeps at least three quarters of the pairs busy (few tokens: the unfused kernels, which
-// split finer, are the better choice).
+// Returns 0 if no admissible S keeps at least three quarters of the pairs busy.  With few tokens (one or two
+// row-strip pairs) a strip is cut into up to 80 segments of one or two ffn tiles: the partial buffer is sized for
+// that at create time (80 splits of at most 1024 rows).
+constexpr int kMaxFusedSegments = 80;
 int fused_segments(int T, int ffn, int rd, size_t part_elems) {
     const int nc = std::max(1, num_sms() / 2), pairs_m = (T + 255) / 256, tiles_n = (ffn + 127) / 128;
-    double best = 0.0;
-    int best_s = 0;
-    for (int S = 1; S <= 16 && S <= tiles_n; ++S) {
-        if ((size_t)S * T * rd > part_elems) break;
+    auto eff_of = [&](int S) {
         const int units = pairs_m * S, rounds = (units + nc - 1) / nc;
-        const double eff = (double)units / ((double)rounds * nc);
-        if (eff > best + 0.03) { best = eff; best_s = S; }   // a finer split must buy 3 % to be worth shorter units
-    }
+        return (double)units / ((double)rounds * nc);
+    };
+    int s_max = std::min(kMaxFusedSegments, tiles_n);
+    while (s_max > 0 && (size_t)s_max * T * rd > part_elems) --s_max;
+    double best = 0.0;
+    for (int S = 1; S <= s_max; ++S) best = std::max(best, eff_of(S));
+    int best_s = 0;
+    for (int S = 1; S <= s_max; ++S)
+        if (eff_of(S) >= best - 0.03) { best_s = S; break; }   // a finer split must buy 3 % to be worth shorter units
     return best >= 0.75 ? best_s : 0;
 }
 
@@ -640,14 +645,16 @@ int launch_convert(const void* in, __half* out, long n, int* flag, cudaStream_t 
 }
 
 int launch_reduce(const float* part, int ksplit, long split_stride, long n, __half* out, cudaStream_t s, float* out32 = nullptr) {
-    int blocks = (int)std::min<long>((n / 4 + 255) / 256, 4 * num_sms());
+    const bool wide = ksplit > 16;   // many splits: eight threads share an output quad (a block covers 128 outputs)
+    int blocks = wide ? (int)std::min<long>((n + 127) / 128, 8 * num_sms()) : (int)std::min<long>((n / 4 + 255) / 256, 4 * num_sms());
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(std::max(blocks, 1)); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, tensorpath::reduce_partials_kernel, part, ksplit, split_stride, n, out, out32));
+    if (wide) CUDA_TRY(cudaLaunchKernelEx(&cfg, tensorpath::reduce_partials_wide_kernel, part, ksplit, split_stride, n, out, out32));
+    else CUDA_TRY(cudaLaunchKernelEx(&cfg, tensorpath::reduce_partials_kernel, part, ksplit, split_stride, n, out, out32));
     return SVDMLP_OK;
 }
 
@@ -916,6 +923,8 @@ int svdmlp_create(svdmlp_t** out, int d, int ffn, int r_gate, int r_up, int r_do
         alloc((void**)&h->H16, (size_t)max_T * ffn * 2);
         alloc((void**)&h->Zd16, (size_t)max_T * r_down * 2);
         h->part_elems = (size_t)16 * max_T * std::max(R, r_down);
+        if (r_gate <= 128 && r_down <= 128)   // the fused gate/up + down-1 kernel cuts short batches into many ffn segments
+            h->part_elems = std::max(h->part_elems, (size_t)kMaxFusedSegments * std::min(max_T, 1024) * r_down);
         alloc((void**)&h->part, h->part_elems * 4);
         alloc((void**)&h->Ug16, (size_t)ffn * r_gate * 2);
         alloc((void**)&h->Uu16, (size_t)ffn * r_up * 2);

@@ -942,6 +942,45 @@ reduce_partials_kernel(const float* __restrict__ part, int ksplit, long split_st
     }
 }
 
+// The same sum for many splits (more than 16).
+// Block = 32 output quads x 8 slices of the splits: with many splits (the fused kernel cuts a short batch into up
+// to 80) a thread that walks all of them alone is bound by L2 latency, so eight threads share an output quad.
+__global__ void __launch_bounds__(256)
+reduce_partials_wide_kernel(const float* __restrict__ part, int ksplit, long split_stride, long n, __half* __restrict__ out,
+                       float* __restrict__ out32) {
+    __shared__ float4 sh[8][32];
+    umma::pdl_launch_dependents();
+    umma::pdl_wait();  // launched with programmatic stream serialization: the partials come from the previous grid
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (long i0 = (long)blockIdx.x * 128; i0 < n; i0 += (long)gridDim.x * 128) {
+        const long i = i0 + tx * 4;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i < n) {
+            for (int k0 = ty; k0 < ksplit; k0 += 32) {   // four loads in flight per thread
+                float4 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    v[j] = (k0 + 8 * j < ksplit) ? *reinterpret_cast<const float4*>(part + (long)(k0 + 8 * j) * split_stride + i)
+                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { s.x += v[j].x; s.y += v[j].y; s.z += v[j].z; s.w += v[j].w; }
+            }
+        }
+        sh[ty][tx] = s;
+        __syncthreads();
+        if (ty == 0 && i < n) {
+#pragma unroll
+            for (int j = 1; j < 8; ++j) { const float4 v = sh[j][tx]; s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
+            uint2 w;
+            w.x = pack_f16(s.x, s.y);
+            w.y = pack_f16(s.z, s.w);
+            *reinterpret_cast<uint2*>(out + i) = w;
+            if (out32 != nullptr) *reinterpret_cast<float4*>(out32 + i) = s;   // the unrounded sum, for a caller that adds shards
+        }
+        __syncthreads();
+    }
+}
+
 // fp32 [n] -> fp16 [n] (n a multiple of 4): a sum of partial Zd shards becomes the operand of the last product.
 __global__ void __launch_bounds__(256)
 f32_to_f16_kernel(const float* __restrict__ in, __half* __restrict__ out, long n) {
