@@ -41,7 +41,7 @@ constexpr int kConsumers = kNW * 32;
 constexpr int kThreads = kConsumers + 32;  // + one producer warp
 constexpr int kSlotBytes = 32768;
 constexpr int kMaxSlots = 8;
-constexpr int kCopiesZd = 4;             // replicated reduction targets of phase B
+constexpr int kCopiesZd = 2;             // replicated reduction targets of phase B
 constexpr int kPanel = 512;              // bytes of a [16 x 16] 16-bit panel
 constexpr int kZdPitch = 32;              // floats per Zd row (token index fastest; T <= 32)
 constexpr int kBarStride = 16;           // u64 words between the barrier words (128 B apart)
