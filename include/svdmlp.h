@@ -72,8 +72,9 @@ int svdmlp_create(svdmlp_t** out, int d, int ffn, int r_gate, int r_up, int r_do
  *   H  = SiLU(Zg Ug^T) .* (Zu Uu^T)     SiLU(g) = g / (1 + e^-g)
  *   Y  = (H Vd^T) Ud^T
  * X bf16; Y bf16 (fp32 with SVDMLP_FLAG_Y_FP32).  Products accumulate in fp32.  1 <= T <= max_T.
- * The kernels are chosen from T alone (weight-streaming kernels for small T, tcgen05 kernels
- * for large T).  Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED, CUDA.
+ * The kernels are chosen from T and the ranks: weight-streaming kernels up to 8 tokens, and up to 32
+ * tokens where the one-kernel decode path fits the shape (ranks 1024: up to 16); tcgen05 kernels
+ * otherwise.  Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED, CUDA.
  */
 int svdmlp_forward(svdmlp_t* h, const void* X, int T, void* Y, void* stream);
 
@@ -111,7 +112,7 @@ int svdmlp_forward_prenorm_residual(svdmlp_t* h, const float* h_in, float* h_out
  *   (the caller sums Zd_out over the shards: an all-reduce)
  *   svdmlp_forward_finish   Y[T, d] = Zd Ud^T,  Zd fp32 [T, r_down] (rounded to fp16 as the product's operand for T > 32)
  * Both are asynchronous on `stream`.  svdmlp_forward_partial followed by svdmlp_forward_finish on the same handle
- * with nothing added in between equals svdmlp_forward.  For T <= 32 the pair runs on the register-streaming
+ * with nothing added in between equals svdmlp_forward.  Where svdmlp_forward streams the weights (T <= 32) the pair runs on the register-streaming
  * decode kernels (the one-kernel decode path cannot stop half way).  Errors as svdmlp_forward.
  */
 int svdmlp_forward_partial(svdmlp_t* h, const void* X, int T, float* Zd_out, void* stream);

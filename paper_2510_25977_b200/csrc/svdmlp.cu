@@ -30,6 +30,7 @@
 
 namespace {
 
+constexpr int kMaxKSplit = 32;             // most K splits of a split-K GEMM (short batches: one tile per SM needs them)
 constexpr int kSkinnyMaxT = 32;            // T <= this uses the weight-streaming kernels
 constexpr int kSmemBudget = 232448 - 1024; // opt-in shared memory per CTA minus alignment slack
 constexpr int kBarrierBytes = 512;
@@ -337,7 +338,7 @@ void plan_gemm(GemmPlan& g, int nb, int bn, bool want_res, bool allow_split, int
         const int base_tiles = m_units * p.tiles_n * batch;
         int ks = std::max(1, units / std::max(1, base_tiles));
         ks = std::min(ks, std::max(1, p.chunks_total / 8));  // keep at least 8 chunks per split
-        ks = std::min(ks, 16);
+        ks = std::min(ks, kMaxKSplit);
         p.ksplit = force_ksplit > 0 ? force_ksplit : ks;   // forced: token slabs of one forward share one partial layout
     }
     p.chunks_per_split = (p.chunks_total + p.ksplit - 1) / p.ksplit;
@@ -509,8 +510,13 @@ dpersist::Shape persist_shape(const svdmlp* h, int T) {
 }
 
 // Number of ring slots the persistent decode kernel gets for T tokens (0: the shape does not fit it).
+int persist_fit(const svdmlp* h, int T, int nt, int nta, bool fused_norm = false, bool x_res = false);
 int persist_slots(const svdmlp* h, int T, int nt, int nta, bool fused_norm = false, bool x_res = false) {
-    if (!h->persist_ok || h->rg != h->ru || T > 8 * nt || (fused_norm && T > 8)) return 0;
+    return h->persist_ok ? persist_fit(h, T, nt, nta, fused_norm, x_res) : 0;
+}
+// The same for a handle whose packed blocks may not exist yet (create-time planning).
+int persist_fit(const svdmlp* h, int T, int nt, int nta, bool fused_norm, bool x_res) {
+    if (h->persist_grid <= 0 || h->rg != h->ru || T > 8 * nt || (fused_norm && T > 8)) return 0;
     const dpersist::Shape sh = persist_shape(h, T);
     if (sh.max_a() > 8 * nta || sh.max_b() > dpersist::kNW || sh.max_d() > dpersist::kNW) return 0;
     const dpersist::Layout L = dpersist::make_layout(sh, nt, nta, fused_norm, x_res);
@@ -841,10 +847,22 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     return SVDMLP_OK;
 }
 
+// Does the persistent decode kernel's shared-memory layout fit for T tokens (whether or not its blocks are packed)?
+bool persist_takes(const svdmlp* h, int T) {
+    if (h->persist_grid <= 0) return false;
+    const int nt = T <= 8 ? 1 : T <= 16 ? 2 : 4;
+    const int nta = persist_shape(h, T).max_a() <= 8 ? 1 : 2;
+    return persist_fit(h, T, nt, nta) > 0;
+}
+
 bool use_skinny(const svdmlp* h, int T) {
     if (h->flags & SVDMLP_FLAG_PATH_SKINNY) return true;
     if (h->flags & SVDMLP_FLAG_PATH_TENSOR) return false;
-    return T <= kSkinnyMaxT || !h->tensor_ok;
+    if (T > kSkinnyMaxT) return !h->tensor_ok;
+    if (T <= 8 || !h->tensor_ok) return true;
+    // 8 < T <= 32: the persistent kernel if it takes the shape; its three-kernel fallback is slower here than the
+    // tcgen05 kernels (T = 32, ranks 1024: 147 us against 48 us)
+    return h->persist_ok && persist_takes(h, T);
 }
 
 int forward_impl(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32, const float* resid, cudaStream_t s,
@@ -918,13 +936,22 @@ int svdmlp_create(svdmlp_t** out, int d, int ffn, int r_gate, int r_up, int r_do
         alloc((void**)&h->Zs, (size_t)h->t_skinny * R * 4);
         alloc((void**)&h->Zds, (size_t)h->t_skinny * r_down * 4);
     }
-    if (h->tensor_ok && (max_T > kSkinnyMaxT || (flags & SVDMLP_FLAG_PATH_TENSOR))) {
+    // The tcgen05 kernels (and their fp16 copies of the second-stage factors) are set up when some T needs them:
+    // above 32 tokens, on request, or between 9 and 32 tokens when the persistent decode kernel cannot take the shape.
+    h->persist_grid = (r_gate == r_up && !(flags & SVDMLP_FLAG_DECODE_REGISTERS)) ? num_sms() : 0;
+    const bool mid_needs_tensor = max_T > 8 && !persist_takes(h, std::min(max_T, kSkinnyMaxT));
+    if (h->tensor_ok && (max_T > kSkinnyMaxT || mid_needs_tensor || (flags & SVDMLP_FLAG_PATH_TENSOR))) {
         alloc((void**)&h->Z16, (size_t)max_T * R * 2);
         alloc((void**)&h->H16, (size_t)max_T * ffn * 2);
         alloc((void**)&h->Zd16, (size_t)max_T * r_down * 2);
-        h->part_elems = (size_t)16 * max_T * std::max(R, r_down);
+        // split-K partials: a split GEMM has at most one tile (128 x 256, or 256 x 256 for a CTA pair) per SM (or
+        // SM pair) over all its splits, which bounds the partial elements whatever T is
+        // (a GEMM that is not split still leaves its one fp32 copy here)
+        const size_t one = (size_t)max_T * std::max(R, r_down);
+        h->part_elems = std::max(one, std::min((size_t)kMaxKSplit * one, (size_t)num_sms() * 128 * 256));
         if (r_gate <= 128 && r_down <= 128)   // the fused gate/up + down-1 kernel cuts short batches into many ffn segments
-            h->part_elems = std::max(h->part_elems, (size_t)kMaxFusedSegments * std::min(max_T, 1024) * r_down);
+            h->part_elems = std::max({h->part_elems, (size_t)kMaxFusedSegments * std::min(max_T, 1024) * r_down,
+                                      (size_t)32 * max_T * r_down});
         alloc((void**)&h->part, h->part_elems * 4);
         alloc((void**)&h->Ug16, (size_t)ffn * r_gate * 2);
         alloc((void**)&h->Uu16, (size_t)ffn * r_up * 2);

@@ -125,6 +125,24 @@ def test_cfg4_rank_sweep(oracle, r, T):
     _gpu.assert_close(Y[rows], _gpu.oracle_rows(oracle, f, X, rows), f"cfg4 r={r} T={T}")
 
 
+@pytest.mark.parametrize("T,r,path", [(16, 1024, "skinny"), (24, 1024, "tensor"), (32, 1024, "tensor"), (32, 512, "skinny")])
+def test_between_9_and_32_tokens_the_path_follows_the_decode_kernels_fit(oracle, T, r, path):
+    """A handle made for at most 32 tokens: where the persistent decode kernel's shared-memory layout does not
+    fit (ranks 1024 above 16 tokens) the tcgen05 kernels run, not the slower three-kernel fallback."""
+    f = inputs.direct_factors(5120, 14336, r, seed=2, device="cuda")
+    X = inputs.activations(T, 5120, seed=2, device="cuda")
+    h = binding.svdmlp_create(*f.tensors(), max_T=T)
+    try:
+        assert binding.svdmlp_path_name(h, T) == path
+        assert binding.svdmlp_path_name(h, 8) == "skinny"
+        Y = binding.svdmlp_forward(h, X)
+        torch.cuda.synchronize()
+        assert binding.svdmlp_last_device_status(h) == 0
+    finally:
+        binding.svdmlp_destroy(h)
+    _gpu.assert_close(Y, _gpu.oracle_rows(oracle, f, X, list(range(T))), f"T={T} r={r} ({path})")
+
+
 @pytest.mark.parametrize("T", [1, 8, 1024])
 def test_cfg5_prenorm_residual_stack(oracle, T):
     d, ffn, r, L = 5120, 13824, 320, 40
