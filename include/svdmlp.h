@@ -185,6 +185,43 @@ int svdlinear_forward_noalloc(const void* X, int T, int in, int out, int r, cons
 int svdmlp_block_aligned_rank(int k, int n, double ratio, int block, double alpha);
 
 /*
+ * Capacity / intensity model of the forward pass on this device: what Section 4.2.1 "Blocking" does with Eq. 10
+ * (arithmetic intensity as a function of the row-strip height B_M) and Eq. 11 (peak on-chip usage) for the
+ * paper's accelerator, restated for the memories of an sm_100 SM.  Host arithmetic only (no CUDA call, usable
+ * without a GPU); it reports the decisions svdmlp_forward takes for the shape, with the numbers behind them.
+ *   strip_rows      B_M: token rows that share one pass over the factor tiles (256: the two CTAs of a pair hold
+ *                   128 rows each and split every factor chunk; 8/16/32 on the weight-streaming path)
+ *   tmem_cols_*     32-bit tensor-memory columns (of 512 per SM) held by the gate/up kernel: the Z strip as packed
+ *                   fp16 A operand (r columns for gate + up, ranks <= 256), the fp32 accumulators of G and Up, and -
+ *                   fused kernel, ranks <= 128 - the fp32 accumulator of Zd
+ *   smem_bytes      shared memory per CTA (of 232448): operand ring, H tile and store staging of that kernel
+ *   flops           2 T r (3 d + 3 ffn)   (Section 3's count for the three factored projections)
+ *   hbm_bytes       factors once + X in + Y out, plus the write and read of H when it is not fused away and is
+ *                   larger than `l2_bytes` (all 16-bit)
+ *   sm_bytes        bytes entering the SMs: Eq. 10's denominator generalised to the MLP - X, Y, Z, Zd, H once each
+ *                   way, and the factors once per row strip:  s [ 2 T d + ceil(T / B_M) 3 r (d + ffn) + ... ]
+ *   intensity_hbm   flops / hbm_bytes;  intensity_sm = flops / sm_bytes (Eq. 10's quantity: it grows with B_M and
+ *                   saturates at 2 r / s per projection)
+ *   ridge_hbm       tensor_tflops / hbm_gbs in FLOP per byte: above it the shape is bound by the tensor pipe
+ *   t_tensor_us, t_hbm_us   flops / tensor_tflops and hbm_bytes / hbm_gbs;  t_floor_us = the larger
+ * path: 0 weight-streaming decode kernels, 1 tcgen05 kernels, 2 tcgen05 kernels with gate/up and the first down
+ * product fused (H never leaves the SM).  tensor_tflops, hbm_gbs: the peaks to model against (<= 0: 1648 TFLOP/s
+ * and 6547 GB/s, measured on a B200); l2_bytes <= 0: 126 MB.  Equal ranks r for the three projections.
+ * Errors: INVALID_ARG (non-positive sizes, NULL out).
+ */
+typedef struct svdmlp_model {
+    int d, ffn, r, T;
+    int path, strip_rows, z_in_tmem;
+    int tmem_cols_strip, tmem_cols_acc, tmem_cols_zd, tmem_cols_total;
+    long smem_bytes;
+    double flops, hbm_bytes, sm_bytes;
+    double intensity_hbm, intensity_sm, ridge_hbm;
+    double t_tensor_us, t_hbm_us, t_floor_us;
+} svdmlp_model_t;
+int svdmlp_model(int d, int ffn, int r, int T, double tensor_tflops, double hbm_gbs, double l2_bytes,
+                 svdmlp_model_t* out);
+
+/*
  * Compression front-end on the device (Section 4.1 with S = I, i.e. without the activation-aware whitening, which
  * needs calibration data: Eq. 3 is then the plain SVD W = U Sigma V^T; Eq. 6-8 fold Sigma into the factors).
  * W[out, in] is a dense fp32 weight on the device; the call writes the factors of the r largest singular values,

@@ -33,9 +33,21 @@ EXPORTS = ["svdmlp_create", "svdmlp_forward", "svdmlp_forward_host", "svdmlp_for
            "svdmlp_compress", "svdmlp_compress_workspace_bytes", "svdmlp_destroy", "svdmlp_strerror",
            "svdmlp_last_device_status", "svdmlp_launch_count", "svdmlp_path_name",
            "svdmlp_profile_enable", "svdmlp_profile_read", "svdmlp_profile_name", "svdmlp_stage_mask",
-           "svdmlp_block_aligned_rank", "svdmlp_selftest_timeout"]
+           "svdmlp_block_aligned_rank", "svdmlp_model", "svdmlp_selftest_timeout"]
 
 _lib = None
+
+
+class Model(ctypes.Structure):
+    """svdmlp_model_t: the capacity / intensity model of one shape (field meanings: include/svdmlp.h)."""
+    _fields_ = [(n, ctypes.c_int) for n in ("d", "ffn", "r", "T", "path", "strip_rows", "z_in_tmem", "tmem_cols_strip",
+                                            "tmem_cols_acc", "tmem_cols_zd", "tmem_cols_total")] + \
+               [("smem_bytes", ctypes.c_long)] + \
+               [(n, ctypes.c_double) for n in ("flops", "hbm_bytes", "sm_bytes", "intensity_hbm", "intensity_sm", "ridge_hbm",
+                                               "t_tensor_us", "t_hbm_us", "t_floor_us")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
 
 
 class SvdMlpError(RuntimeError):
@@ -92,6 +104,8 @@ def lib() -> ctypes.CDLL:
         L.svdmlp_path_name.argtypes = [vp, ci]
         L.svdmlp_block_aligned_rank.restype = ci
         L.svdmlp_block_aligned_rank.argtypes = [ci, ci, ctypes.c_double, ci, ctypes.c_double]
+        L.svdmlp_model.restype = ci
+        L.svdmlp_model.argtypes = [ci, ci, ci, ci, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.POINTER(Model)]
         L.svdmlp_selftest_timeout.restype = ci
         L.svdmlp_selftest_timeout.argtypes = [vp, cu, vp]
         L.svdmlp_stage_mask.restype = ci
@@ -211,6 +225,12 @@ def svdmlp_block_aligned_rank(k: int, n: int, ratio: float, block: int, alpha: f
     if r < 0:
         raise SvdMlpError(r, "svdmlp_block_aligned_rank")
     return r
+
+
+def svdmlp_model(d: int, ffn: int, r: int, T: int, tensor_tflops: float = 0.0, hbm_gbs: float = 0.0, l2_bytes: float = 0.0) -> dict:
+    m = Model()
+    _check(lib().svdmlp_model(d, ffn, r, T, tensor_tflops, hbm_gbs, l2_bytes, ctypes.byref(m)), "svdmlp_model")
+    return m.as_dict()
 
 
 def svdlinear_workspace_bytes(T: int, n_in: int, n_out: int, r: int) -> int:

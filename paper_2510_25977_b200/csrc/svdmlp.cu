@@ -307,6 +307,26 @@ int down1_tile_width(int rd) {
     return (rd <= 128 || pad256 * 4 > pad128 * 5) ? 128 : 256;
 }
 
+// Gate/up at ranks above 256: do 256-wide pair tiles quantise onto the clusters about as well as 128-wide ones?
+bool gateup_wide_pays(int tiles_m, int ffn) {
+    const long nc = num_sms() / 2, pm = (tiles_m + 1) / 2;
+    const long t256 = pm * ((ffn + 255) / 256), t128 = pm * ((ffn + 127) / 128);
+    const long rounds256 = (t256 + nc - 1) / nc, rounds128 = (t128 + nc - 1) / nc;
+    return 2 * rounds256 * 100 <= rounds128 * 108;
+}
+
+// Elements of the split-K partial buffer for a handle made for max_T tokens.
+// A split GEMM has at most one tile (128 x 256, or 256 x 256 for a CTA pair) per SM (or SM pair) over all its
+// splits, which bounds the partial elements whatever T is; a GEMM that is not split still leaves its one fp32
+// copy here; the fused gate/up + down-1 kernel cuts short batches into many ffn segments.
+size_t part_elems_for(int max_T, int R, int r_gate, int r_down) {
+    const size_t one = (size_t)max_T * std::max(R, r_down);
+    size_t n = std::max(one, std::min((size_t)kMaxKSplit * one, (size_t)num_sms() * 128 * 256));
+    if (r_gate <= 128 && r_down <= 128)
+        n = std::max({n, (size_t)kMaxFusedSegments * std::min(max_T, 1024) * r_down, (size_t)32 * max_T * r_down});
+    return n;
+}
+
 // Fill the shape-dependent part of a plan (tensor maps are set by the caller).
 // want_res: keep the A strip resident if it fits.  allow_split: use split-K to fill the machine.
 void plan_gemm(GemmPlan& g, int nb, int bn, bool want_res, bool allow_split, int M, int N, int K, int batch,
@@ -785,10 +805,8 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     // the tile count quantises onto the clusters about as well as 128-wide tiles do
     bool wide = false;
     if (!ts && g.pair && !g.ares && h->rg == h->ru && h->rg > 256 && !(h->flags & SVDMLP_FLAG_NO_WIDE_GATEUP)) {
-        const long nc = num_sms() / 2, pm = (g.p.tiles_m + 1) / 2;
-        const long t256 = pm * ((h->ffn + 255) / 256), t128 = pm * ((h->ffn + 127) / 128);
-        const long rounds256 = (t256 + nc - 1) / nc, rounds128 = (t128 + nc - 1) / nc;
-        wide = 2 * rounds256 * 100 <= rounds128 * 108;
+        const long nc = num_sms() / 2, t256 = (long)((g.p.tiles_m + 1) / 2) * ((h->ffn + 255) / 256);
+        wide = gateup_wide_pays(g.p.tiles_m, h->ffn);
         if (wide) {
             g.p.tiles_n = (h->ffn + 255) / 256;
             g.grid = 2 * (int)std::min<long>(t256, nc);
@@ -900,6 +918,72 @@ int svdmlp_block_aligned_rank(int k, int n, double ratio, int block, double alph
     return r > 0x7fffffffLL ? SVDMLP_ERR_INVALID_ARG : (int)r;
 }
 
+int svdmlp_model(int d, int ffn, int r, int T, double tensor_tflops, double hbm_gbs, double l2_bytes, svdmlp_model_t* out) {
+    if (out == nullptr || d <= 0 || ffn <= 0 || r <= 0 || T <= 0) return SVDMLP_ERR_INVALID_ARG;
+    if (!(tensor_tflops > 0.0)) tensor_tflops = 1648.0;
+    if (!(hbm_gbs > 0.0)) hbm_gbs = 6547.0;
+    if (!(l2_bytes > 0.0)) l2_bytes = 126e6;
+    svdmlp_model_t m;
+    memset(&m, 0, sizeof(m));
+    m.d = d; m.ffn = ffn; m.r = r; m.T = T;
+    // the routing of svdmlp_forward, on a handle that holds the shape only
+    svdmlp* h = new (std::nothrow) svdmlp();
+    if (h == nullptr) return SVDMLP_ERR_NOMEM;
+    memset(h, 0, sizeof(*h));
+    h->d = d; h->ffn = ffn; h->rg = h->ru = h->rd = r; h->max_T = T;
+    h->persist_grid = num_sms(); h->persist_ok = true; h->tensor_ok = true; h->stage_mask = ~0u;
+    h->part_elems = part_elems_for(T, 2 * r, r, r);
+    const bool stream_weights = use_skinny(h, T);
+    const int S = stream_weights ? 0 : fused_plan(h, T);
+    delete h;
+    const double s2 = 2.0;  // bytes per element of X, Y, the factors and the 16-bit intermediates
+    m.flops = 2.0 * T * r * (3.0 * d + 3.0 * ffn);
+    const double factors = s2 * 3.0 * r * ((double)d + ffn), h_bytes = s2 * T * (double)ffn;
+    if (stream_weights) {
+        m.path = 0;
+        m.strip_rows = T <= 8 ? 8 : T <= 16 ? 16 : 32;
+        // mma.sync path: no tensor memory; shared memory = the whole opt-in budget (ring slots take what the
+        // activations leave)
+        m.smem_bytes = (long)kPersistSmemBudget;
+    } else {
+        using namespace tensorpath;
+        m.path = S > 0 ? 2 : 1;
+        const int tiles_m = (T + BM - 1) / BM;
+        m.strip_rows = tiles_m >= 2 ? 2 * BM : BM;
+        GemmPlan g;
+        plan_gemm(g, 2, 128, true, false, T, ffn, r, 1, true, true);
+        const bool ts = g.pair && g.ares && r <= 256;
+        const bool wide = !ts && g.pair && !g.ares && r > 256 && gateup_wide_pays(g.p.tiles_m, ffn);
+        if (S > 0) {          // strips [0, 128), Zd [128, 256), G [256, 384), Up [384, 512)
+            m.z_in_tmem = 1; m.tmem_cols_strip = 128; m.tmem_cols_zd = 128; m.tmem_cols_acc = 256;
+            m.smem_bytes = kFuSmemBytes;
+        } else if (ts) {      // gate strip [0, 128), up strip [128, 256), G [256, 384), Up [384, 512)
+            m.z_in_tmem = 1; m.tmem_cols_strip = 256; m.tmem_cols_acc = 256;
+            m.smem_bytes = kTsSmemBytes;
+        } else if (wide) {    // two 256-column accumulators, both operands streamed
+            m.tmem_cols_acc = 512;
+            m.smem_bytes = kWideSmemBytes;
+        } else {              // 128-wide tiles, G and Up double-buffered; the Z strip in shared memory if it fits
+            m.tmem_cols_acc = 512;
+            m.smem_bytes = (long)g.smem;
+        }
+    }
+    m.tmem_cols_total = m.tmem_cols_strip + m.tmem_cols_acc + m.tmem_cols_zd;
+    const bool h_fused = m.path != 1;   // decode and fused kernels keep H on the SM
+    m.hbm_bytes = factors + 2.0 * s2 * T * (double)d + ((!h_fused && h_bytes > l2_bytes) ? 2.0 * h_bytes : 0.0);
+    const double strips = (double)((T + m.strip_rows - 1) / m.strip_rows);
+    // X and Y once; the factors once per row strip; Z (2r) and Zd (r) written and read once; H written and read once
+    m.sm_bytes = 2.0 * s2 * T * (double)d + strips * factors + 2.0 * s2 * T * 3.0 * r + (h_fused ? 0.0 : 2.0 * h_bytes);
+    m.intensity_hbm = m.flops / m.hbm_bytes;
+    m.intensity_sm = m.flops / m.sm_bytes;
+    m.ridge_hbm = tensor_tflops * 1e3 / hbm_gbs;
+    m.t_tensor_us = m.flops / (tensor_tflops * 1e6);
+    m.t_hbm_us = m.hbm_bytes / (hbm_gbs * 1e3);
+    m.t_floor_us = std::max(m.t_tensor_us, m.t_hbm_us);
+    *out = m;
+    return SVDMLP_OK;
+}
+
 int svdmlp_create(svdmlp_t** out, int d, int ffn, int r_gate, int r_up, int r_down, const void* Ug, const void* Vg,
                   const void* Uu, const void* Vu, const void* Ud, const void* Vd, int max_T, unsigned flags,
                   void* stream) {
@@ -944,14 +1028,7 @@ int svdmlp_create(svdmlp_t** out, int d, int ffn, int r_gate, int r_up, int r_do
         alloc((void**)&h->Z16, (size_t)max_T * R * 2);
         alloc((void**)&h->H16, (size_t)max_T * ffn * 2);
         alloc((void**)&h->Zd16, (size_t)max_T * r_down * 2);
-        // split-K partials: a split GEMM has at most one tile (128 x 256, or 256 x 256 for a CTA pair) per SM (or
-        // SM pair) over all its splits, which bounds the partial elements whatever T is
-        // (a GEMM that is not split still leaves its one fp32 copy here)
-        const size_t one = (size_t)max_T * std::max(R, r_down);
-        h->part_elems = std::max(one, std::min((size_t)kMaxKSplit * one, (size_t)num_sms() * 128 * 256));
-        if (r_gate <= 128 && r_down <= 128)   // the fused gate/up + down-1 kernel cuts short batches into many ffn segments
-            h->part_elems = std::max({h->part_elems, (size_t)kMaxFusedSegments * std::min(max_T, 1024) * r_down,
-                                      (size_t)32 * max_T * r_down});
+        h->part_elems = part_elems_for(max_T, R, r_gate, r_down);
         alloc((void**)&h->part, h->part_elems * 4);
         alloc((void**)&h->Ug16, (size_t)ffn * r_gate * 2);
         alloc((void**)&h->Uu16, (size_t)ffn * r_up * 2);
