@@ -144,6 +144,20 @@ typedef struct svdlinear svdlinear_t; /* opaque */
 int svdlinear_create(svdlinear_t** out_handle, int in, int out, int r, const void* U, const void* V, int max_T,
                      void* stream);
 int svdlinear_apply(svdlinear_t* h, const void* X, int T, void* Y, void* stream);
+/*
+ * The same with the layout flags of Algorithm 2's XUV_Kernel (is_XT: the input arrives pre-transposed; req_OT:
+ * the output is wanted transposed), so that a caller whose neighbouring operators work on transposed activations
+ * needs no transpose pass of its own:
+ *   SVDLINEAR_X_TRANSPOSED   X is X^T[in, T] (row-major, T contiguous)
+ *   SVDLINEAR_Y_TRANSPOSED   Y is written as Y^T[out, T]
+ * With either flag T must be a multiple of 8 (16-byte row pitch).  For T > 32 neither costs a pass over memory:
+ * X^T tiles are loaded as they are and multiplied as an MN-major operand, and the epilogue stores transposed
+ * tiles.  For T <= 32 the operand (at most 32 rows) passes through a scratch copy.  layout = 0 is svdlinear_apply.
+ * Errors: as svdlinear_apply; ALIGNMENT also for T not a multiple of 8 with a flag set.
+ */
+#define SVDLINEAR_X_TRANSPOSED 0x1u
+#define SVDLINEAR_Y_TRANSPOSED 0x2u
+int svdlinear_apply_layout(svdlinear_t* h, const void* X, int T, void* Y, unsigned layout, void* stream);
 int svdlinear_destroy(svdlinear_t* h);
 
 /*

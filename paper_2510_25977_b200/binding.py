@@ -29,7 +29,7 @@ FLAG_NO_FUSED_DOWN1 = 0x1000
 EXPORTS = ["svdmlp_create", "svdmlp_forward", "svdmlp_forward_host", "svdmlp_forward_prenorm_residual",
            "svdmlp_forward_partial", "svdmlp_forward_finish",
            "svdlinear_forward", "svdlinear_workspace_bytes", "svdlinear_forward_noalloc",
-           "svdlinear_create", "svdlinear_apply", "svdlinear_destroy",
+           "svdlinear_create", "svdlinear_apply", "svdlinear_apply_layout", "svdlinear_destroy",
            "svdmlp_compress", "svdmlp_compress_workspace_bytes", "svdmlp_destroy", "svdmlp_strerror",
            "svdmlp_last_device_status", "svdmlp_launch_count", "svdmlp_path_name",
            "svdmlp_profile_enable", "svdmlp_profile_read", "svdmlp_profile_name", "svdmlp_stage_mask",
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.svdlinear_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, vp, vp, ci, vp]
         L.svdlinear_apply.restype = ci
         L.svdlinear_apply.argtypes = [vp, vp, ci, vp, vp]
+        L.svdlinear_apply_layout.restype = ci
+        L.svdlinear_apply_layout.argtypes = [vp, vp, ci, vp, cu, vp]
         L.svdlinear_destroy.restype = ci
         L.svdlinear_destroy.argtypes = [vp]
         L.svdlinear_workspace_bytes.restype = ctypes.c_size_t
@@ -280,6 +282,20 @@ def svdlinear_apply(h: LinearHandle, X, Y=None, stream=None) -> torch.Tensor:
     if Y is None:
         Y = torch.empty((X.shape[0], h.n_out), dtype=torch.bfloat16, device=X.device)
     _check(lib().svdlinear_apply(h.ptr, _ptr(X), X.shape[0], _ptr(Y), _stream(stream)), "svdlinear_apply")
+    return Y
+
+
+X_TRANSPOSED, Y_TRANSPOSED = 0x1, 0x2
+
+
+def svdlinear_apply_layout(h: LinearHandle, X, layout: int, Y=None, stream=None) -> torch.Tensor:
+    """svdlinear_apply with Algorithm 2's layout flags: X_TRANSPOSED: X is X^T[in, T]; Y_TRANSPOSED: the result is
+    Y^T[out, T]."""
+    T = X.shape[1] if layout & X_TRANSPOSED else X.shape[0]
+    if Y is None:
+        shape = (h.n_out, T) if layout & Y_TRANSPOSED else (T, h.n_out)
+        Y = torch.empty(shape, dtype=torch.bfloat16, device=X.device)
+    _check(lib().svdlinear_apply_layout(h.ptr, _ptr(X), T, _ptr(Y), layout, _stream(stream)), "svdlinear_apply_layout")
     return Y
 
 

@@ -119,6 +119,21 @@ int make_map_f32(CUtensorMap* m, const void* base, long rows, long cols, long ld
     return r == CUDA_SUCCESS ? SVDMLP_OK : SVDMLP_ERR_CUDA;
 }
 
+// Row-major 16-bit matrix [rows, cols] written in boxes of [64 rows, 32 columns] without swizzle: the transposed
+// output C^T[N, M] of a GEMM whose epilogue stages [64 n][32 m] tiles.
+int make_map_t(CUtensorMap* m, const void* base, long rows, long cols, long ld) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return SVDMLP_ERR_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {32, 64};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SVDMLP_OK : SVDMLP_ERR_CUDA;
+}
+
 // ---- tensor-path launch helper ----------------------------------------------------------------
 struct GemmPlan {
     int nb, bn;
@@ -384,6 +399,7 @@ void plan_gemm(GemmPlan& g, int nb, int bn, bool want_res, bool allow_split, int
         g.pair = true;
     }
     p.split_stride = 0; p.batch_col_off = 0; p.resid = nullptr;
+    p.a_mn = 0; p.c_t = 0;
     if (!(g.pair && !g.ares)) p.cps = 1;
 }
 
@@ -1451,8 +1467,9 @@ struct svdlinear {
     float* f32; __half *z16, *u16;
     bool u16_ok;
     CUtensorMap mV, mU, mZ, mZc;
-    const void* x_ptr; int x_T; CUtensorMap mX;
-    const void* y_ptr; int y_T; CUtensorMap mYc;
+    const void* x_ptr; int x_T; unsigned x_layout; CUtensorMap mX;
+    const void* y_ptr; int y_T; unsigned y_layout; CUtensorMap mYc;
+    uint16_t *xt, *yt;   // [32, in] and [32, out] scratch: transposed layouts at T <= 32
 };
 
 namespace {
@@ -1461,7 +1478,7 @@ namespace {
 // leave through TMA stores.  Z[T, r] passes through global memory in fp16 (L2-resident at these sizes).
 int lin_tensor_run(const CUtensorMap& mX, const CUtensorMap& mV, const CUtensorMap& mU, const CUtensorMap& mZ,
                    const CUtensorMap& mZc, const CUtensorMap& mYc, float* f32, __half* z16, void* Y, int T, int in,
-                   int out, int r, cudaStream_t s) {
+                   int out, int r, cudaStream_t s, unsigned layout = 0) {
     using namespace tensorpath;
     int rc;
     const bool pr = T > BM;
@@ -1470,6 +1487,7 @@ int lin_tensor_run(const CUtensorMap& mX, const CUtensorMap& mV, const CUtensorM
     plan_gemm(g, 1, bn, false, true, T, r, in, 1, true, pr);
     g.p.tmA[0] = mX; g.p.tmA[1] = mX; g.p.tmB[0] = mV; g.p.tmB[1] = mV; g.p.tmC = mZc;
     g.p.a_fmt = umma::kFmtBF16; g.p.b_fmt = umma::kFmtBF16; g.p.status = nullptr;
+    g.p.a_mn = (layout & SVDLINEAR_X_TRANSPOSED) ? 1 : 0;   // mX then maps X^T[in, T]: the tile is an MN-major operand
     if (g.p.ksplit > 1) {
         g.p.c_tma = 0;  // fp32 partials are stored directly
         g.p.C = f32; g.p.ldc = r; g.p.split_stride = (long)T * r; g.p.out_mode = OUT_F32;
@@ -1483,6 +1501,7 @@ int lin_tensor_run(const CUtensorMap& mX, const CUtensorMap& mV, const CUtensorM
     g.p.tmA[0] = mZ; g.p.tmA[1] = mZ; g.p.tmB[0] = mU; g.p.tmB[1] = mU; g.p.tmC = mYc;
     g.p.a_fmt = umma::kFmtF16; g.p.b_fmt = umma::kFmtF16; g.p.status = nullptr;
     g.p.C = Y; g.p.ldc = out; g.p.out_mode = OUT_BF16;
+    g.p.c_t = (layout & SVDLINEAR_Y_TRANSPOSED) ? 1 : 0;    // mYc then maps Y^T[out, T]
     return launch_gemm(g, s);
 }
 }  // namespace
@@ -1569,6 +1588,8 @@ int svdlinear_create(svdlinear_t** out_h, int in, int out, int r, const void* U,
     h->in = in; h->out = out; h->r = r; h->max_T = max_T; h->U = U; h->V = V;
     h->ws_bytes = svdlinear_workspace_bytes(max_T, in, out, r);
     if (cudaMalloc(&h->ws, h->ws_bytes) != cudaSuccess) { cudaGetLastError(); delete h; return SVDMLP_ERR_NOMEM; }
+    if (cudaMalloc((void**)&h->xt, (size_t)kSkinnyMaxT * (in + out) * 2) != cudaSuccess) { cudaGetLastError(); svdlinear_destroy(h); return SVDMLP_ERR_NOMEM; }
+    h->yt = h->xt + (size_t)kSkinnyMaxT * in;
     h->f32 = reinterpret_cast<float*>(h->ws);
     h->z16 = reinterpret_cast<__half*>(reinterpret_cast<char*>(h->ws) + ((lin_f32_elems(max_T, r) * 4 + 255) & ~(size_t)255));
     h->u16 = h->z16 + (((size_t)max_T * r * 2 + 255) & ~(size_t)255) / 2;
@@ -1592,22 +1613,46 @@ int svdlinear_create(svdlinear_t** out_h, int in, int out, int r, const void* U,
 }
 
 int svdlinear_apply(svdlinear_t* h, const void* X, int T, void* Y, void* stream) {
+    return svdlinear_apply_layout(h, X, T, Y, 0u, stream);
+}
+
+int svdlinear_apply_layout(svdlinear_t* h, const void* X, int T, void* Y, unsigned layout, void* stream) {
     if (h == nullptr || X == nullptr || Y == nullptr || T <= 0 || T > h->max_T) return SVDMLP_ERR_INVALID_ARG;
+    if (layout & ~(SVDLINEAR_X_TRANSPOSED | SVDLINEAR_Y_TRANSPOSED)) return SVDMLP_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(Y)) return SVDMLP_ERR_ALIGNMENT;
+    if (layout != 0 && (T & 7)) return SVDMLP_ERR_ALIGNMENT;   // rows of X^T / Y^T are T elements: 16-byte pitch
+    const bool xt = layout & SVDLINEAR_X_TRANSPOSED, yt = layout & SVDLINEAR_Y_TRANSPOSED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (T <= kSkinnyMaxT)   // weight-streaming kernels read the bf16 factors as they are
-        return svdlinear_forward(X, T, h->in, h->out, h->r, h->U, h->V, Y, h->ws, h->ws_bytes, stream);
+    if (T <= kSkinnyMaxT) {
+        // weight-streaming kernels read the bf16 factors as they are; they take row-major X and Y, so a
+        // transposed operand (at most 32 rows) passes through a scratch copy
+        const void* Xr = X;
+        void* Yr = Y;
+        if (xt) {
+            tensorpath::transpose16_kernel<<<dim3((T + 31) / 32, (h->in + 31) / 32), 256, 0, s>>>((const uint16_t*)X, h->in, T, h->xt);
+            Xr = h->xt;
+        }
+        if (yt) Yr = h->yt;
+        int rc = svdlinear_forward(Xr, T, h->in, h->out, h->r, h->U, h->V, Yr, h->ws, h->ws_bytes, stream);
+        if (rc != SVDMLP_OK) return rc;
+        if (yt) tensorpath::transpose16_kernel<<<dim3((h->out + 31) / 32, (T + 31) / 32), 256, 0, s>>>(h->yt, T, h->out, (uint16_t*)Y);
+        CUDA_TRY(cudaGetLastError());
+        return SVDMLP_OK;
+    }
     if (!h->u16_ok) return SVDMLP_ERR_UNSUPPORTED;
     int rc;
-    if (h->x_ptr != X || h->x_T != T) {
-        if ((rc = make_map(&h->mX, X, T, h->in, h->in, tensorpath::BM)) != SVDMLP_OK) return rc;
-        h->x_ptr = X; h->x_T = T;
+    if (h->x_ptr != X || h->x_T != T || h->x_layout != (layout & SVDLINEAR_X_TRANSPOSED)) {
+        // X^T[in, T]: boxes of [64 k][64 tokens]; X[T, in]: boxes of [128 tokens][64 k]
+        rc = xt ? make_map(&h->mX, X, h->in, T, T, 64) : make_map(&h->mX, X, T, h->in, h->in, tensorpath::BM);
+        if (rc != SVDMLP_OK) return rc;
+        h->x_ptr = X; h->x_T = T; h->x_layout = layout & SVDLINEAR_X_TRANSPOSED;
     }
-    if (h->y_ptr != Y || h->y_T != T) {
-        if ((rc = make_map(&h->mYc, Y, T, h->out, h->out, 32)) != SVDMLP_OK) return rc;
-        h->y_ptr = Y; h->y_T = T;
+    if (h->y_ptr != Y || h->y_T != T || h->y_layout != (layout & SVDLINEAR_Y_TRANSPOSED)) {
+        rc = yt ? make_map_t(&h->mYc, Y, h->out, T, T) : make_map(&h->mYc, Y, T, h->out, h->out, 32);
+        if (rc != SVDMLP_OK) return rc;
+        h->y_ptr = Y; h->y_T = T; h->y_layout = layout & SVDLINEAR_Y_TRANSPOSED;
     }
-    return lin_tensor_run(h->mX, h->mV, h->mU, h->mZ, h->mZc, h->mYc, h->f32, h->z16, Y, T, h->in, h->out, h->r, s);
+    return lin_tensor_run(h->mX, h->mV, h->mU, h->mZ, h->mZc, h->mYc, h->f32, h->z16, Y, T, h->in, h->out, h->r, s, layout);
 }
 
 int svdlinear_destroy(svdlinear_t* h) {
@@ -1615,6 +1660,7 @@ int svdlinear_destroy(svdlinear_t* h) {
     cudaDeviceSynchronize();
     cudaGetLastError();
     if (h->ws != nullptr) cudaFree(h->ws);
+    if (h->xt != nullptr) cudaFree(h->xt);
     delete h;
     return SVDMLP_OK;
 }

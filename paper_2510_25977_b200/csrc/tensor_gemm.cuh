@@ -49,6 +49,9 @@ struct GemmParams {
     int a_fmt, b_fmt;    // umma::kFmtF16 / kFmtBF16
     const float* resid;  // optional fp32 [M, ldc] added to an OUT_F32 result (residual connection)
     int* status;         // device status word (written on timeout)
+    // Layout flags of the XUV operator (Algorithm 2's is_XT / req_OT); streaming one-branch kernels only.
+    int a_mn;            // 1: A is given transposed, A^T[K, M]: tmA has boxes [64 k][64 m], the tile is an MN-major operand
+    int c_t;             // 1: the 16-bit TMA-store epilogue writes C^T[N, M]: tmC has boxes [64 n][32 m], no swizzle
 };
 
 __device__ __forceinline__ float fast_silu(float g) {
@@ -207,8 +210,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                             if (ARES) {
                                 umma::tma_load_2d(st, &p.tmB[NB == 2 ? sl : tc.z], &full[stage], c * BK, tc.n * BN);
                             } else {
-                                for (int b = 0; b < NB; ++b)
-                                    umma::tma_load_2d(st + b * kABytes, &p.tmA[NB == 2 ? b : tc.z], &full[stage], c * BK, tc.m * BM);
+                                for (int b = 0; b < NB; ++b) {
+                                    if (p.a_mn) {  // two boxes [64 k][64 m] of A^T
+                                        umma::tma_load_2d(st + b * kABytes, &p.tmA[NB == 2 ? b : tc.z], &full[stage], tc.m * BM, c * BK);
+                                        umma::tma_load_2d(st + b * kABytes + kABytes / 2, &p.tmA[NB == 2 ? b : tc.z], &full[stage], tc.m * BM + 64, c * BK);
+                                    } else {
+                                        umma::tma_load_2d(st + b * kABytes, &p.tmA[NB == 2 ? b : tc.z], &full[stage], c * BK, tc.m * BM);
+                                    }
+                                }
                                 for (int b = 0; b < NB; ++b)
                                     umma::tma_load_2d(st + NB * kABytes + b * B_BYTES, &p.tmB[NB == 2 ? b : tc.z],
                                                       &full[stage], c * BK, tc.n * BN);
@@ -222,7 +231,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         }
     } else if (warp == 1) {
         {  // ---------------- MMA issuer: warp-uniform waits, one elected lane issues ----------------
-            const uint32_t idesc = umma::make_idesc(p.a_fmt, p.b_fmt, BM, BN);
+            const uint32_t idesc = umma::make_idesc(p.a_fmt, p.b_fmt, BM, BN) | (p.a_mn ? umma::kIdescAMnMajor : 0u);
+            const uint64_t a_step = p.a_mn ? 128 : 2;  // descriptor units of 16 B per K = 16: two 8-k groups, or 32 B inside the swizzle atom
             int stage = 0, cur_m = -1, acc = 0;
             uint32_t phase = 0, a_phase = 0, acc_phase0 = 0, acc_phase1 = 0;
             bool ok = true;
@@ -258,14 +268,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                                 uint64_t ad[NB], bd[NB];
 #pragma unroll
                                 for (int b = 0; b < NB; ++b) {
-                                    ad[b] = umma::smem_desc_sw128(umma::smem_u32(st + b * kABytes));
+                                    ad[b] = p.a_mn ? umma::smem_desc_sw128_mn(umma::smem_u32(st + b * kABytes), kABytes / 2)
+                                                   : umma::smem_desc_sw128(umma::smem_u32(st + b * kABytes));
                                     bd[b] = umma::smem_desc_sw128(umma::smem_u32(st + NB * kABytes + b * B_BYTES));
                                 }
 #pragma unroll
                                 for (int kk = 0; kk < BK / 16; ++kk)
 #pragma unroll
                                     for (int b = 0; b < NB; ++b)
-                                        umma::mma_f16_ss(dcol + b * BN, ad[b] + 2 * kk, bd[b] + 2 * kk, idesc,
+                                        umma::mma_f16_ss(dcol + b * BN, ad[b] + a_step * kk, bd[b] + 2 * kk, idesc,
                                                          (c > c_begin) || (kk > 0));
                             }
                             umma::mma_commit(&empty[stage]);
@@ -413,15 +424,25 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     }
                     umma::bulk_wait_read0();  // the previous store has finished reading the staging tile
                     __syncwarp();
+                    if (p.c_t) {   // transposed tile [64 columns][32 rows]: a column's 32 rows are one 64-byte line
+                        uint16_t* st16 = reinterpret_cast<uint16_t*>(my_stage);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            st16[(2 * i) * 32 + lane] = (uint16_t)(packed[i] & 0xffffu);
+                            st16[(2 * i + 1) * 32 + lane] = (uint16_t)(packed[i] >> 16);
+                        }
+                    } else {
 #pragma unroll
                     for (int ch = 0; ch < 8; ++ch)
                         *reinterpret_cast<uint4*>(my_stage + lane * 128 + ((ch ^ (lane & 7)) << 4)) =
                             make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
+                    }
                     umma::fence_proxy_async_smem();
                     __syncwarp();
                     const int col = tc.n * BN + c0;
                     if (lane == 0 && col < p.N && tc.m * BM + q * 32 < p.M) {
-                        umma::tma_store_2d(&p.tmC, my_stage, col + (int)(tc.z * p.batch_col_off), tc.m * BM + q * 32);
+                        if (p.c_t) umma::tma_store_2d(&p.tmC, my_stage, tc.m * BM + q * 32, col + (int)(tc.z * p.batch_col_off));
+                        else umma::tma_store_2d(&p.tmC, my_stage, col + (int)(tc.z * p.batch_col_off), tc.m * BM + q * 32);
                         umma::bulk_commit();
                     }
                 }
@@ -616,7 +637,12 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
 #pragma unroll
                                 for (int b = 0; b < NB; ++b) {
                                     unsigned char* sb = st + j * SLOT_BYTES + b * (kABytes + HB_BYTES);
-                                    umma::tma_load_2d_pair(sb, &p.tmA[NB == 2 ? b : z], bar, (c + j) * BK, m * BM);
+                                    if (p.a_mn) {  // two boxes [64 k][64 m] of A^T
+                                        umma::tma_load_2d_pair(sb, &p.tmA[NB == 2 ? b : z], bar, m * BM, (c + j) * BK);
+                                        umma::tma_load_2d_pair(sb + kABytes / 2, &p.tmA[NB == 2 ? b : z], bar, m * BM + 64, (c + j) * BK);
+                                    } else {
+                                        umma::tma_load_2d_pair(sb, &p.tmA[NB == 2 ? b : z], bar, (c + j) * BK, m * BM);
+                                    }
                                     umma::tma_load_2d_pair(sb + kABytes, &p.tmB[NB == 2 ? b : z], bar, (c + j) * BK,
                                                            n * BN + (int)rank * (BN / 2));
                                 }
@@ -630,7 +656,8 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
     } else if (warp == 1 || (NISS == 2 && warp == 10)) {
         if (leader) {  // ---------------- MMA issuer(s) (leader CTA only) ----------------
             const int bsel = (warp == 1) ? 0 : 1;  // with two issuers: the branch this one feeds
-            const uint32_t idesc = umma::make_idesc(p.a_fmt, p.b_fmt, 2 * BM, BN);
+            const uint32_t idesc = umma::make_idesc(p.a_fmt, p.b_fmt, 2 * BM, BN) | (p.a_mn ? umma::kIdescAMnMajor : 0u);
+            const uint64_t a_step = p.a_mn ? 128 : 2;
             int stage = 0, cur_mp = -1, acc = 0;
             uint32_t phase = 0, a_phase = 0, acc_phase0 = 0, acc_phase1 = 0;
             bool ok = true;
@@ -670,12 +697,13 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                                     const unsigned char* b_ptr = ARES ? st + b * HB_BYTES : a_ptr + kABytes;
                                     // Descriptors step by 32 bytes (2 in address units of 16) along K inside the
                                     // swizzle atom; shared memory is below 256 KiB, so the 14-bit field never carries.
-                                    const uint64_t ad = umma::smem_desc_sw128(umma::smem_u32(a_ptr));
+                                    const uint64_t ad = (!ARES && p.a_mn) ? umma::smem_desc_sw128_mn(umma::smem_u32(a_ptr), kABytes / 2)
+                                                                          : umma::smem_desc_sw128(umma::smem_u32(a_ptr));
                                     const uint64_t bd = umma::smem_desc_sw128(umma::smem_u32(b_ptr));
                                     const uint32_t dcol = tmem_base + acc * ACC_COLS + br * BN;
 #pragma unroll
                                     for (int kk = 0; kk < BK / 16; ++kk)
-                                        umma::mma_f16_ss_pair(dcol, ad + 2 * kk, bd + 2 * kk, idesc,
+                                        umma::mma_f16_ss_pair(dcol, ad + a_step * kk, bd + 2 * kk, idesc,
                                                               (c + j > c_begin) || (kk > 0));
                                 }
                             umma::mma_commit_pair(&empty[stage]);
@@ -833,15 +861,25 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                     }
                     umma::bulk_wait_read0();  // the previous store has finished reading the staging tile
                     __syncwarp();
+                    if (p.c_t) {   // transposed tile [64 columns][32 rows]: a column's 32 rows are one 64-byte line
+                        uint16_t* st16 = reinterpret_cast<uint16_t*>(my_stage);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            st16[(2 * i) * 32 + lane] = (uint16_t)(packed[i] & 0xffffu);
+                            st16[(2 * i + 1) * 32 + lane] = (uint16_t)(packed[i] >> 16);
+                        }
+                    } else {
 #pragma unroll
                     for (int ch = 0; ch < 8; ++ch)
                         *reinterpret_cast<uint4*>(my_stage + lane * 128 + ((ch ^ (lane & 7)) << 4)) =
                             make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
+                    }
                     umma::fence_proxy_async_smem();
                     __syncwarp();
                     const int col = n * BN + c0;
                     if (lane == 0 && col < p.N && m * BM + q * 32 < p.M) {
-                        umma::tma_store_2d(&p.tmC, my_stage, col + (int)(z * p.batch_col_off), m * BM + q * 32);
+                        if (p.c_t) umma::tma_store_2d(&p.tmC, my_stage, m * BM + q * 32, col + (int)(z * p.batch_col_off));
+                        else umma::tma_store_2d(&p.tmC, my_stage, col + (int)(z * p.batch_col_off), m * BM + q * 32);
                         umma::bulk_commit();
                     }
                 }
@@ -897,6 +935,19 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
     }
     umma::cluster_sync();  // neither CTA's shared memory or TMEM goes away while the partner may still use it
     if (warp == 1) { umma::tc_fence_after_sync(); umma::tmem_dealloc_pair(tmem_base, TMEM_COLS); }
+}
+
+// out[c, r] = in[r, c] for a 16-bit matrix in[rows, cols] (32 x 32 tiles through shared memory).  Used only for
+// the transposed layouts of the XUV operator at T <= 32, where the weight-streaming kernels run.
+__global__ void __launch_bounds__(256)
+transpose16_kernel(const uint16_t* __restrict__ in, int rows, int cols, uint16_t* __restrict__ out) {
+    __shared__ uint16_t tile[32][33];
+    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32, tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int i = ty; i < 32; i += 8)
+        if (r0 + i < rows && c0 + tx < cols) tile[i][tx] = in[(long)(r0 + i) * cols + c0 + tx];
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8)
+        if (c0 + i < cols && r0 + tx < rows) out[(long)(c0 + i) * rows + r0 + tx] = tile[tx][i];
 }
 
 // Exact re-encoding of bf16 weights as fp16 (tcgen05 kind::f16 wants A and B in the same 16-bit

@@ -242,6 +242,20 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr) {
     d |= (uint64_t)2 << 61;
     return d;
 }
+// The same for an MN-major operand tile: rows of 64 16-bit elements along M (or N), one row per k, as TMA writes
+// a box [64 k][64 m] of a matrix whose contiguous dimension is M.  8-row (8 k) groups are 1024 B apart (stride
+// byte offset); the next 64 elements along M start `lbo_bytes` further on (leading byte offset: the next box).
+// A K = 16 MMA covers two 8-k groups, so consecutive MMAs advance the start address by 2048 B.
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t smem_addr, uint32_t lbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+constexpr uint32_t kIdescAMnMajor = 1u << 15;  // instruction descriptor: A is MN-major ("transposed")
 // Instruction descriptor for kind::f16: fp32 accumulate, K-major A and B.
 //   bits 4-5 D format (1 = f32) | 7-9 A format | 10-12 B format (0 = f16, 1 = bf16)
 //   15/16 A/B major (0 = K) | 17-22 N >> 3 | 24-28 M >> 4

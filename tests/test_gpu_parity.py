@@ -393,6 +393,46 @@ def test_svdlinear_handle(oracle, T, n_in, n_out, r):
     binding.svdlinear_destroy(h)
 
 
+@pytest.mark.parametrize("layout", [1, 2, 3])
+@pytest.mark.parametrize("T,n_in,n_out,r", [(8, 264, 696, 40), (32, 264, 696, 40), (40, 264, 696, 40), (128, 264, 696, 40),
+                                            (136, 264, 696, 40), (520, 264, 696, 40), (1024, 2048, 4096, 256)])
+def test_svdlinear_transposed_layouts(oracle, T, n_in, n_out, r, layout):
+    """Algorithm 2's is_XT / req_OT: X given as X^T[in, T] and / or Y wanted as Y^T[out, T].  Every element is compared
+    (the oracle on X itself; a layout flag changes where elements sit, not their values), on shapes with ragged
+    tiles in every dimension, on both sides of the 32-token and 128-token path boundaries."""
+    V = inputs.normal_tensor(14, 0, (r, n_in), scale=n_in ** -0.5, device="cuda")
+    U = inputs.normal_tensor(14, 1, (n_out, r), scale=r ** -0.5, device="cuda")
+    X = inputs.activations(T, n_in, seed=14 + T, device="cuda")
+    h = binding.svdlinear_create(U, V, max_T=T)
+    try:
+        Xin = X.t().contiguous() if layout & binding.X_TRANSPOSED else X
+        out = binding.svdlinear_apply_layout(h, Xin, layout)
+        plain = binding.svdlinear_apply(h, X)
+        torch.cuda.synchronize()
+    finally:
+        binding.svdlinear_destroy(h)
+    assert out.shape == ((n_out, T) if layout & binding.Y_TRANSPOSED else (T, n_out))
+    Y = out.t() if layout & binding.Y_TRANSPOSED else out
+    rows = list(range(T)) if T <= 520 else inputs.sample_rows(T, max_rows=48)
+    _gpu.assert_close(Y[rows], oracle.svdlinear(X[rows], U, V), f"layout={layout} T={T}")
+    if T > 32 and not layout & binding.X_TRANSPOSED:
+        assert torch.equal(Y.contiguous(), plain)      # the same accumulators, stored elsewhere
+
+
+def test_svdlinear_layout_argument_checks():
+    V = inputs.normal_tensor(15, 0, (16, 64), scale=0.1, device="cuda")
+    U = inputs.normal_tensor(15, 1, (64, 16), scale=0.1, device="cuda")
+    h = binding.svdlinear_create(U, V, max_T=64)
+    L = binding.lib()
+    X = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
+    Y = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
+    assert L.svdlinear_apply_layout(h.ptr, X.data_ptr(), 12, Y.data_ptr(), 1, None) == -3     # T not a multiple of 8
+    assert L.svdlinear_apply_layout(h.ptr, X.data_ptr(), 16, Y.data_ptr(), 4, None) == -1     # unknown flag
+    assert L.svdlinear_apply_layout(h.ptr, X.data_ptr(), 12, Y.data_ptr(), 0, None) == 0
+    torch.cuda.synchronize()
+    binding.svdlinear_destroy(h)
+
+
 def test_svdlinear_handle_reports_factors_outside_the_fp16_range():
     """A factor value beyond 65504 cannot be re-encoded for the large-T kernels: the handle says so (status -2) for
     T > 32 instead of returning inf/NaN, and still serves small T on the bf16 kernels."""
