@@ -119,6 +119,32 @@ int svdmlp_forward_partial(svdmlp_t* h, const void* X, int T, float* Zd_out, voi
 int svdmlp_forward_finish(svdmlp_t* h, const float* Zd, int T, void* Y, void* stream);
 
 /*
+ * The same pair with the exchange done by the library's own kernels instead of a collective library (Figure 4's
+ * AllReduce, on the narrow Zd): every rank pushes its partial into its slot of every peer's receive buffer with
+ * plain peer stores and raises one flag per peer; the finishing call waits (bounded) for the flags of the step and
+ * sums the slots.  Set-up, by the caller, once: on every rank a receive buffer of svdmlp_tp_recv_bytes(G, max_T,
+ * r_down) bytes and G 64-bit flag words, ZEROED, both mapped into every peer (peer access, IPC or symmetric
+ * memory); `peers` lists them by rank as this rank addresses them.  Steps are numbered 1, 2, 3, ... and every rank
+ * calls push(step) then gather(step), on one stream, for each step in turn (the two-deep buffering relies on it).
+ *   svdmlp_forward_partial_push    Zd_g of this shard -> slot `rank` of every rank's buffer; flags[rank] = step
+ *   svdmlp_forward_finish_gather   waits for flags[0..G) >= step, Zd = sum of the slots, Y = Zd Ud^T.
+ *     recv, flags: THIS rank's buffer and flag words.  A wait that outlasts the limit (2 s unless changed through
+ *     svdmlp_tp_wait_limit_ns of svdmlp_bench.h) sets the status word (svdmlp_last_device_status: -7), leaves Y
+ *     unspecified and returns normally: nothing spins without bound.
+ * G <= 8.  Errors: as svdmlp_forward_partial / svdmlp_forward_finish; INVALID_ARG also for step 0 or a bad rank.
+ */
+typedef struct svdmlp_tp_peers {
+    int world, rank;                 /* G and this rank's index */
+    float* recv[8];                  /* recv[p]: rank p's receive buffer, as addressed from this rank */
+    unsigned long long* flags[8];    /* flags[p]: rank p's G flag words */
+} svdmlp_tp_peers_t;
+size_t svdmlp_tp_recv_bytes(int world, int max_T, int r_down);
+int svdmlp_forward_partial_push(svdmlp_t* h, const void* X, int T, const svdmlp_tp_peers_t* peers,
+                                unsigned long long step, void* stream);
+int svdmlp_forward_finish_gather(svdmlp_t* h, float* recv, const unsigned long long* flags, int world,
+                                 unsigned long long step, int T, void* Y, void* stream);
+
+/*
  * The paper's XUV operator (Section 4.2.1):  Y[T, out] = (X[T, in] V^T) U^T  with U[out, r],
  * V[r, in]; X, U, V, Y bf16.  `workspace` is caller-owned device scratch of at least
  * svdlinear_workspace_bytes(T, in, out, r) bytes, 256-byte aligned; its contents are

@@ -52,6 +52,9 @@ int svdmlp_stage_mask(svdmlp_t* h, unsigned mask);
  * gate/up and the first down product in one kernel: ranks up to 128). */
 const char* svdmlp_path_name(const svdmlp_t* h, int T);
 
+/* Test aid: how long svdmlp_forward_finish_gather waits for its peers' flags before it gives up (default 2 s). */
+int svdmlp_tp_wait_limit_ns(svdmlp_t* h, unsigned long long limit_ns);
+
 #ifdef __cplusplus
 }
 #endif

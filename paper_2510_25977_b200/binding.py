@@ -28,6 +28,7 @@ FLAG_NO_FUSED_DOWN1 = 0x1000
 
 EXPORTS = ["svdmlp_create", "svdmlp_forward", "svdmlp_forward_host", "svdmlp_forward_prenorm_residual",
            "svdmlp_forward_partial", "svdmlp_forward_finish",
+           "svdmlp_forward_partial_push", "svdmlp_forward_finish_gather", "svdmlp_tp_recv_bytes", "svdmlp_tp_wait_limit_ns",
            "svdlinear_forward", "svdlinear_workspace_bytes", "svdlinear_forward_noalloc",
            "svdlinear_create", "svdlinear_apply", "svdlinear_apply_layout", "svdlinear_destroy",
            "svdmlp_compress", "svdmlp_compress_workspace_bytes", "svdmlp_destroy", "svdmlp_strerror",
@@ -36,6 +37,11 @@ EXPORTS = ["svdmlp_create", "svdmlp_forward", "svdmlp_forward_host", "svdmlp_for
            "svdmlp_block_aligned_rank", "svdmlp_model", "svdmlp_selftest_timeout"]
 
 _lib = None
+
+
+class TpPeers(ctypes.Structure):
+    """svdmlp_tp_peers_t: the receive buffers and flag words of all ranks, as addressed from this rank."""
+    _fields_ = [("world", ctypes.c_int), ("rank", ctypes.c_int), ("recv", ctypes.c_void_p * 8), ("flags", ctypes.c_void_p * 8)]
 
 
 class Model(ctypes.Structure):
@@ -106,6 +112,14 @@ def lib() -> ctypes.CDLL:
         L.svdmlp_path_name.argtypes = [vp, ci]
         L.svdmlp_block_aligned_rank.restype = ci
         L.svdmlp_block_aligned_rank.argtypes = [ci, ci, ctypes.c_double, ci, ctypes.c_double]
+        L.svdmlp_tp_recv_bytes.restype = ctypes.c_size_t
+        L.svdmlp_tp_recv_bytes.argtypes = [ci, ci, ci]
+        L.svdmlp_forward_partial_push.restype = ci
+        L.svdmlp_forward_partial_push.argtypes = [vp, vp, ci, ctypes.POINTER(TpPeers), ctypes.c_ulonglong, vp]
+        L.svdmlp_forward_finish_gather.restype = ci
+        L.svdmlp_forward_finish_gather.argtypes = [vp, vp, vp, ci, ctypes.c_ulonglong, ci, vp, vp]
+        L.svdmlp_tp_wait_limit_ns.restype = ci
+        L.svdmlp_tp_wait_limit_ns.argtypes = [vp, ctypes.c_ulonglong]
         L.svdmlp_model.restype = ci
         L.svdmlp_model.argtypes = [ci, ci, ci, ci, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.POINTER(Model)]
         L.svdmlp_selftest_timeout.restype = ci
@@ -220,6 +234,35 @@ def svdmlp_forward_prenorm_residual(h: Handle, h_in: torch.Tensor, h_out: torch.
     _check(lib().svdmlp_forward_prenorm_residual(h.ptr, _ptr(h_in), _ptr(h_out), h_in.shape[0], eps, _stream(stream)),
            "svdmlp_forward_prenorm_residual")
     return h_out
+
+
+def svdmlp_tp_recv_bytes(world: int, max_T: int, r_down: int) -> int:
+    return int(lib().svdmlp_tp_recv_bytes(world, max_T, r_down))
+
+
+def tp_peers(rank: int, recv_ptrs, flag_ptrs) -> TpPeers:
+    p = TpPeers()
+    p.world, p.rank = len(recv_ptrs), rank
+    for i, (r, f) in enumerate(zip(recv_ptrs, flag_ptrs)):
+        p.recv[i], p.flags[i] = r, f
+    return p
+
+
+def svdmlp_forward_partial_push(h: Handle, X, peers: TpPeers, step: int, stream=None):
+    _check(lib().svdmlp_forward_partial_push(h.ptr, _ptr(X), X.shape[0], ctypes.byref(peers), step, _stream(stream)),
+           "svdmlp_forward_partial_push")
+
+
+def svdmlp_forward_finish_gather(h: Handle, recv, flags, world: int, step: int, T: int, Y=None, stream=None):
+    if Y is None:
+        Y = torch.empty((T, h.d), dtype=torch.float32 if h.flags & FLAG_Y_FP32 else torch.bfloat16, device=recv.device)
+    _check(lib().svdmlp_forward_finish_gather(h.ptr, _ptr(recv), _ptr(flags), world, step, T, _ptr(Y), _stream(stream)),
+           "svdmlp_forward_finish_gather")
+    return Y
+
+
+def svdmlp_tp_wait_limit_ns(h: Handle, ns: int):
+    _check(lib().svdmlp_tp_wait_limit_ns(h.ptr, ns), "svdmlp_tp_wait_limit_ns")
 
 
 def svdmlp_block_aligned_rank(k: int, n: int, ratio: float, block: int, alpha: float = 0.5) -> int:

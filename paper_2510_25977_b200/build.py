@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsvdmlp.so")
 SOURCES = ["svdmlp.cu"]
-HEADERS = ["skinny.cuh", "umma.cuh", "tensor_gemm.cuh", "gateup_ts.cuh", "mlp_fused_ts.cuh", "gateup_wide.cuh", "compress.cuh", "decode_persistent.cuh", os.path.join("..", "..", "include", "svdmlp.h"),
+HEADERS = ["skinny.cuh", "umma.cuh", "tensor_gemm.cuh", "gateup_ts.cuh", "mlp_fused_ts.cuh", "gateup_wide.cuh", "compress.cuh", "tp_exchange.cuh", "decode_persistent.cuh", os.path.join("..", "..", "include", "svdmlp.h"),
            os.path.join("..", "..", "include", "svdmlp_bench.h")]
 
 

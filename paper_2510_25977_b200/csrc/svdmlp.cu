@@ -25,6 +25,7 @@
 #include "tensor_gemm.cuh"
 #include "gateup_ts.cuh"
 #include "mlp_fused_ts.cuh"
+#include "tp_exchange.cuh"
 #include "gateup_wide.cuh"
 #include "compress.cuh"
 
@@ -442,6 +443,8 @@ struct svdmlp {
     const void* x_ptr; int x_T; CUtensorMap mX;
     CUtensorMap mHc, mYc; const void* y_ptr; int y_T, y_f32;
     float* zd_out32;                  // svdmlp_forward_partial: where the fp32 Zd of this call goes (else NULL)
+    unsigned int* tp_counter;         // block counter of the tensor-parallel push kernel (zero between launches)
+    unsigned long long tp_limit_ns;   // how long the tensor-parallel gather waits for its peers
     SlabPlan slabs;                   // token slabs of the gate/up -> down-1 pair for the last T seen (maps cached)
     CUtensorMap mUg64, mUu64, mUd64;  // half-tile boxes [64 rows, 64 columns] for the CTA-pair kernels
     CUtensorMap mVg64, mVu64, mVg128, mVu128, mVdHalf;  // half-tile boxes of the first-GEMM factors
@@ -1033,6 +1036,8 @@ int svdmlp_create(svdmlp_t** out, int d, int ffn, int r_gate, int r_up, int r_do
     };
     alloc((void**)&h->status_dev, sizeof(int));
     alloc((void**)&h->gridbar, kGridbarBytes);
+    alloc((void**)&h->tp_counter, 256);
+    h->tp_limit_ns = 2000000000ull;
     if (h->t_skinny > 0) {
         alloc((void**)&h->Zs, (size_t)h->t_skinny * R * 4);
         alloc((void**)&h->Zds, (size_t)h->t_skinny * r_down * 4);
@@ -1056,7 +1061,8 @@ int svdmlp_create(svdmlp_t** out, int d, int ffn, int r_gate, int r_up, int r_do
     }
     if (!ok) { svdmlp_destroy(h); return SVDMLP_ERR_NOMEM; }
     bool cuda_ok = cudaMemsetAsync(h->status_dev, 0, sizeof(int), s) == cudaSuccess &&
-                   cudaMemsetAsync(h->gridbar, 0, kGridbarBytes, s) == cudaSuccess;
+                   cudaMemsetAsync(h->gridbar, 0, kGridbarBytes, s) == cudaSuccess &&
+                   cudaMemsetAsync(h->tp_counter, 0, 256, s) == cudaSuccess;
     if (h->Zs) cuda_ok = cuda_ok && cudaMemsetAsync(h->Zs, 0, (size_t)h->t_skinny * R * 4, s) == cudaSuccess;
     if (h->Zds) cuda_ok = cuda_ok && cudaMemsetAsync(h->Zds, 0, (size_t)h->t_skinny * r_down * 4, s) == cudaSuccess;
     if (cuda_ok && h->tensor_ok) {
@@ -1306,12 +1312,66 @@ int svdmlp_forward_finish(svdmlp_t* h, const float* Zd, int T, void* Y, void* st
     return rc;
 }
 
+// ---- tensor-parallel forward with the exchange done by the library's own kernels (tp_exchange.cuh) -----------
+size_t svdmlp_tp_recv_bytes(int G, int max_T, int r_down) {
+    if (G <= 0 || G > tpx::kMaxRanks || max_T <= 0 || r_down <= 0) return 0;
+    return (size_t)2 * G * max_T * r_down * sizeof(float);
+}
+
+int svdmlp_forward_partial_push(svdmlp_t* h, const void* X, int T, const svdmlp_tp_peers_t* peers, unsigned long long step,
+                                void* stream) {
+    if (h == nullptr || peers == nullptr || step == 0) return SVDMLP_ERR_INVALID_ARG;
+    const int G = peers->world, rank = peers->rank;
+    if (G <= 0 || G > tpx::kMaxRanks || rank < 0 || rank >= G) return SVDMLP_ERR_INVALID_ARG;
+    tpx::Peers pp;
+    for (int p = 0; p < G; ++p) {
+        if (peers->recv[p] == nullptr || peers->flags[p] == nullptr) return SVDMLP_ERR_INVALID_ARG;
+        if (!aligned16(peers->recv[p]) || (reinterpret_cast<uintptr_t>(peers->flags[p]) & 7)) return SVDMLP_ERR_ALIGNMENT;
+        pp.recv[p] = peers->recv[p]; pp.flags[p] = peers->flags[p];
+    }
+    const long slot = (long)h->max_T * h->rd, slot_off = ((long)(step & 1ull) * G + rank) * slot;
+    // this rank's partial goes straight into its own slot of its own receive buffer ...
+    const int rc = svdmlp_forward_partial(h, X, T, peers->recv[rank] + slot_off, stream);
+    if (rc != SVDMLP_OK) return rc;
+    // ... and from there to the same slot of every peer; the flags follow the data
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const long n = (long)T * h->rd;
+    const int blocks = (int)std::max<long>(1, std::min<long>((n / 4 + 255) / 256, 2L * num_sms()));
+    tpx::push_kernel<<<blocks, 256, 0, s>>>(peers->recv[rank] + slot_off, n, pp, G, rank, slot_off, step, h->tp_counter);
+    CUDA_TRY(cudaGetLastError());
+    h->launches += 1;
+    return SVDMLP_OK;
+}
+
+int svdmlp_forward_finish_gather(svdmlp_t* h, float* recv, const unsigned long long* flags, int G, unsigned long long step,
+                                 int T, void* Y, void* stream) {
+    if (h == nullptr || recv == nullptr || flags == nullptr || Y == nullptr || step == 0 || G <= 0 || G > tpx::kMaxRanks ||
+        T <= 0 || T > h->max_T)
+        return SVDMLP_ERR_INVALID_ARG;
+    if (!aligned16(recv) || (reinterpret_cast<uintptr_t>(flags) & 7)) return SVDMLP_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const long slot = (long)h->max_T * h->rd, n = (long)T * h->rd;
+    float* base = recv + (long)(step & 1ull) * G * slot;
+    const int blocks = (int)std::max<long>(1, std::min<long>((n / 4 + 255) / 256, 2L * num_sms()));
+    // the sum replaces slot 0 of this step's buffer (each element is read, then written, by one thread)
+    tpx::gather_sum_kernel<<<blocks, 256, 0, s>>>(base, flags, G, step, n, slot, base, h->status_dev, h->tp_limit_ns);
+    CUDA_TRY(cudaGetLastError());
+    h->launches += 1;
+    return svdmlp_forward_finish(h, base, T, Y, stream);
+}
+
+int svdmlp_tp_wait_limit_ns(svdmlp_t* h, unsigned long long limit_ns) {
+    if (h == nullptr || limit_ns == 0) return SVDMLP_ERR_INVALID_ARG;
+    h->tp_limit_ns = limit_ns;
+    return SVDMLP_OK;
+}
+
 int svdmlp_destroy(svdmlp_t* h) {
     if (h == nullptr) return SVDMLP_OK;
     cudaDeviceSynchronize();
     cudaGetLastError();
     void* bufs[] = {h->Zs, h->Zds, h->Z16, h->H16, h->Zd16, h->part, h->Ug16, h->Uu16, h->Vd16, h->Ud16,
-                    h->Xn, h->Xdev, h->Ydev, h->status_dev, h->gridbar,
+                    h->Xn, h->Xdev, h->Ydev, h->status_dev, h->gridbar, h->tp_counter,
                     h->pA, h->pB, h->pVdp, h->pUdp, h->Zp, h->Zdp};
     for (void* b : bufs)
         if (b != nullptr) cudaFree(b);

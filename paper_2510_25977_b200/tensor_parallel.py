@@ -31,3 +31,34 @@ def forward(binding, handle, X, dist=None, Y=None, stream=None):
     if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(Zd)
     return binding.svdmlp_forward_finish(handle, Zd, Y, stream=stream)
+
+
+class Exchange:
+    """Receive buffers and flag words for the library's own exchange (svdmlp_forward_partial_push /
+    svdmlp_forward_finish_gather).  `ranks_on_this_device` > 0 builds the buffers of ALL ranks on the current device:
+    the single-GPU form used by the tests, where the ranks' calls run one after the other on one stream (a push
+    never waits, so nothing can block).  Across GPUs every process allocates its own pair and passes the peers'
+    mapped addresses (peer access, IPC handles or symmetric memory) to `binding.tp_peers` itself."""
+
+    def __init__(self, binding, world: int, max_T: int, r_down: int, device="cuda"):
+        import torch
+        n = binding.svdmlp_tp_recv_bytes(world, max_T, r_down) // 4
+        self.world = world
+        self.recv = [torch.zeros(n, dtype=torch.float32, device=device) for _ in range(world)]
+        self.flags = [torch.zeros(world, dtype=torch.int64, device=device) for _ in range(world)]
+        self.step = 0
+        self._binding = binding
+
+    def peers(self, rank: int):
+        return self._binding.tp_peers(rank, [t.data_ptr() for t in self.recv], [t.data_ptr() for t in self.flags])
+
+
+def forward_all_ranks_on_one_device(binding, handles, X, ex: Exchange, stream=None):
+    """One tensor-parallel step with every rank's handle on this device: all pushes, then all gathers.  Returns the G
+    outputs (they are equal up to nothing: every rank sums the same G slots in the same order)."""
+    ex.step += 1
+    T = X.shape[0]
+    for g, h in enumerate(handles):
+        binding.svdmlp_forward_partial_push(h, X, ex.peers(g), ex.step, stream=stream)
+    return [binding.svdmlp_forward_finish_gather(h, ex.recv[g], ex.flags[g], ex.world, ex.step, T, stream=stream)
+            for g, h in enumerate(handles)]

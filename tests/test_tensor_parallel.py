@@ -99,3 +99,73 @@ def test_sharded_handles_on_one_gpu(oracle, T, world):
     _gpu.assert_close(Y3, ref, "plain forward after the halves")
     for hh in handles + [h]:
         binding.svdmlp_destroy(hh)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("T", [8, 27, 300])
+@pytest.mark.parametrize("world", [2, 4])
+def test_exchange_by_the_librarys_own_kernels(oracle, T, world):
+    """svdmlp_forward_partial_push / svdmlp_forward_finish_gather with every rank's buffers on this one device: the
+    ranks' calls run one after the other on one stream, so no kernel ever waits for a later one.  Three steps in a
+    row use both halves of the two-deep receive buffers; every rank must produce the same bits (all sum the same
+    slots in the same order) and match the oracle."""
+    import _gpu
+    from paper_2510_25977_b200 import binding
+    _gpu.require_gpu()
+    d, ffn, r = 512, 1408, 64
+    f = inputs.direct_factors(d, ffn, r, seed=6, device="cuda")
+    handles = [binding.svdmlp_create(*tp.shard_factors(*f.tensors(), world, g), max_T=T) for g in range(world)]
+    ex = tp.Exchange(binding, world, T, r)
+    try:
+        for step in range(3):
+            X = inputs.activations(T, d, seed=60 + step, device="cuda")
+            Ys = tp.forward_all_ranks_on_one_device(binding, handles, X, ex)
+            torch.cuda.synchronize()
+            for h in handles:
+                assert binding.svdmlp_last_device_status(h) == 0
+            for Y in Ys[1:]:
+                assert torch.equal(Y, Ys[0])
+            _gpu.assert_close(Ys[0], oracle.svdmlp(X, *f.tensors()), f"exchange x{world}, T={T}, step {step + 1}")
+        assert all(int(v) == 3 for fl in ex.flags for v in fl.tolist())
+    finally:
+        for h in handles:
+            binding.svdmlp_destroy(h)
+
+
+@pytest.mark.gpu
+def test_exchange_gather_gives_up_when_a_peer_never_pushes():
+    """Failure detection without a fault: rank 1 never pushes step 1, rank 0's gather waits out its (shortened) limit,
+    sets the status word and returns; the context stays usable and a later complete step succeeds."""
+    import _gpu
+    from paper_2510_25977_b200 import binding
+    _gpu.require_gpu()
+    d, ffn, r, T, world = 256, 768, 32, 8, 2
+    f = inputs.direct_factors(d, ffn, r, seed=7, device="cuda")
+    X = inputs.activations(T, d, seed=7, device="cuda")
+    handles = [binding.svdmlp_create(*tp.shard_factors(*f.tensors(), world, g), max_T=T) for g in range(world)]
+    ex = tp.Exchange(binding, world, T, r)
+    try:
+        binding.svdmlp_tp_wait_limit_ns(handles[0], 20_000_000)          # 20 ms
+        binding.svdmlp_forward_partial_push(handles[0], X, ex.peers(0), 1)
+        binding.svdmlp_forward_finish_gather(handles[0], ex.recv[0], ex.flags[0], world, 1, T)
+        torch.cuda.synchronize()
+        assert binding.svdmlp_last_device_status(handles[0]) == -7
+        assert binding.svdmlp_last_device_status(handles[0]) == 0        # cleared by the read
+        ex.step = 1                                                      # step 1 is lost; both ranks go on with step 2
+        Ys = tp.forward_all_ranks_on_one_device(binding, handles, X, ex)
+        torch.cuda.synchronize()
+        assert binding.svdmlp_last_device_status(handles[0]) == 0 and torch.equal(Ys[0], Ys[1])
+        assert torch.isfinite(Ys[0].float()).all()
+    finally:
+        for h in handles:
+            binding.svdmlp_destroy(h)
+
+
+def test_exchange_argument_checks():
+    from paper_2510_25977_b200 import binding, build
+    build.build()
+    L = binding.lib()
+    assert L.svdmlp_tp_recv_bytes(2, 8, 32) == 2 * 2 * 8 * 32 * 4
+    assert L.svdmlp_tp_recv_bytes(9, 8, 32) == 0 and L.svdmlp_tp_recv_bytes(0, 8, 32) == 0
+    assert L.svdmlp_forward_partial_push(None, None, 1, None, 1, None) == -1
+    assert L.svdmlp_forward_finish_gather(None, None, None, 2, 1, 1, None, None) == -1
