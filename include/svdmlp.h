@@ -74,7 +74,10 @@ int svdmlp_create(svdmlp_t** out, int d, int ffn, int r_gate, int r_up, int r_do
  * X bf16; Y bf16 (fp32 with SVDMLP_FLAG_Y_FP32).  Products accumulate in fp32.  1 <= T <= max_T.
  * The kernels are chosen from T and the ranks: weight-streaming kernels up to 8 tokens, and up to 32
  * tokens where the one-kernel decode path fits the shape (ranks 1024: up to 16); tcgen05 kernels
- * otherwise.  Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED, CUDA.
+ * otherwise.  Reproducibility: the tcgen05 kernels sum in a fixed order, so repeated calls on the same inputs give
+ * the same bits; the weight-streaming kernels reduce Zd over the ffn slices with fp32 atomic adds, whose order is
+ * not fixed, so their outputs can differ between calls in the last bits (fp32 rounding of a 148-term sum, far
+ * inside the bf16 rounding of Y for most elements).  Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED, CUDA.
  */
 int svdmlp_forward(svdmlp_t* h, const void* X, int T, void* Y, void* stream);
 
