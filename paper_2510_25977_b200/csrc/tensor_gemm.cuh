@@ -178,6 +178,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     // Programmatic dependent launch: everything above overlapped the previous kernel's tail; its
     // results (our A operand, and buffers we overwrite) may only be touched after this wait.
     umma::pdl_launch_dependents();
+    // The B operands are weights, which no earlier kernel writes: the first tile's chunks are requested into L2
+    // before this grid waits for its predecessor, so their first (HBM) touch overlaps the predecessor's tail.
+    if (warp == 0 && lane == 0 && tile_begin < tile_end) {
+        const TileCoord tc = decode_tile<ARES>(p, tile_begin);
+        const int c_begin = tc.ks * p.chunks_per_split, c_end = min(p.chunks_total, c_begin + min(p.chunks_per_split, 16));
+        for (int b = 0; b < NB; ++b)
+            for (int c = c_begin; c < c_end; ++c)
+                umma::tma_prefetch_2d(&p.tmB[NB == 2 ? b : tc.z], c * BK, tc.n * BN);
+    }
     umma::pdl_wait();
 
     if (warp == 0) {
