@@ -281,30 +281,54 @@ expand_kernel(const float* __restrict__ A, int T, int r, const __nv_bfloat16* __
         }
 }
 
-// RMSNorm with unit weight, fp32 in, bf16 out: one block per token row.
+// RMSNorm with unit weight, fp32 in, bf16 out: one block per token row.  Rows of up to 8192 elements are held in
+// registers (all loads issued before the first use, one pass over memory); longer rows are read twice.
+// Launched with programmatic stream serialization: the row is only read after the preceding kernel has finished.
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const float* __restrict__ h, int d, float eps, __nv_bfloat16* __restrict__ out) {
     __shared__ float red[8];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const float* row = h + (long)blockIdx.x * d;
+    __nv_bfloat16* o = out + (long)blockIdx.x * d;
+    const bool in_regs = d <= 8 * 256 * 4;
+    float4 v[8];
     float ss = 0.f;
-    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
-        float4 v = *reinterpret_cast<const float4*>(row + i);
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    if (in_regs) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = (j * 256 + threadIdx.x) * 4;
+            v[j] = (i < d) ? *reinterpret_cast<const float4*>(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) ss += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
+    } else {
+        for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+            const float4 w = *reinterpret_cast<const float4*>(row + i);
+            ss += w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
+        }
     }
-    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
     __syncthreads();
     float tot = 0.f;
     for (int w = 0; w < 8; ++w) tot += red[w];
     const float inv = rsqrtf(tot / (float)d + eps);
-    __nv_bfloat16* o = out + (long)blockIdx.x * d;
-    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
-        float4 v = *reinterpret_cast<const float4*>(row + i);
-        __nv_bfloat162 a = __floats2bfloat162_rn(v.x * inv, v.y * inv), b = __floats2bfloat162_rn(v.z * inv, v.w * inv);
+    auto emit = [&](int i, const float4& w) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(w.x * inv, w.y * inv), b = __floats2bfloat162_rn(w.z * inv, w.w * inv);
         uint2 pk;
         pk.x = *reinterpret_cast<uint32_t*>(&a);
         pk.y = *reinterpret_cast<uint32_t*>(&b);
         *reinterpret_cast<uint2*>(o + i) = pk;
+    };
+    if (in_regs) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = (j * 256 + threadIdx.x) * 4;
+            if (i < d) emit(i, v[j]);
+        }
+    } else {
+        for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) emit(i, *reinterpret_cast<const float4*>(row + i));
     }
 }
 

@@ -1231,7 +1231,13 @@ int svdmlp_forward_prenorm_residual(svdmlp_t* h, const float* h_in, float* h_out
     }
     if (h->stage_mask & 16u) {
         ProfScope ps(h, "rmsnorm", s);
-        skinny::rmsnorm_kernel<<<T, 256, 0, s>>>(h_in, h->d, eps, h->Xn);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(T); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        CUDA_TRY(cudaLaunchKernelEx(&cfg, skinny::rmsnorm_kernel, h_in, h->d, eps, h->Xn));
     }
     CUDA_TRY(cudaGetLastError());
     h->launches += 1;
