@@ -763,6 +763,20 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
             decode(t, mp, n, ks, z);
             const int m = 2 * mp + (int)rank;
             if (t + 1 < tile_end) prefetch_resid(t + 1);
+            // fp32 + residual epilogue: the residual of a 32-column group is loaded one group ahead (the first
+            // group's before the accumulator is even complete), so its latency hides behind the mainloop and
+            // behind the previous group's staging and store instead of standing in front of every group.
+            float4 rs[8];
+            auto load_rs = [&](int c0n) {
+                const int rrow0 = m * BM + q * 32 + (lane >> 3), rcol = n * BN + c0n + 4 * (lane & 7);
+                if (p.resid != nullptr && rcol + 4 <= p.N) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        rs[i] = (rrow0 + 4 * i < p.M) ? *reinterpret_cast<const float4*>(p.resid + (long)(rrow0 + 4 * i) * p.ldc + rcol)
+                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            };
+            if (p.c_tma && p.out_mode == OUT_F32) load_rs(half * (BN / 2));
             ok = umma::mbar_wait_warp(&tfull[acc], acc ? acc_phase1 : acc_phase0, abort_flag);
             if (!ok) break;
             umma::tc_fence_after_sync();
@@ -784,17 +798,10 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                     const int col = n * BN + c0;
                     // Residual: the warp reads the [32 x 32] tile cooperatively (lane = 16-byte chunk (lane & 7) of
                     // rows 4 i + lane / 8: every load instruction covers four whole 128-byte lines) and adds it to
-                    // the staged tile in shared memory. The loads are issued before the TMEM wait; one row per lane
-                    // (32 lines per instruction) took about 2000 cycles per group.
-                    float4 rs[8];
-                    const int rrow0 = m * BM + q * 32 + (lane >> 3), rcol = col + 4 * (lane & 7);
+                    // the staged tile in shared memory (one row per lane, 32 lines per instruction, took about 2000
+                    // cycles per group).  rs holds this group's values, loaded one group ago.
+                    const int rcol = col + 4 * (lane & 7);
                     const bool radd = p.resid != nullptr && rcol + 4 <= p.N;
-                    if (radd) {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            rs[i] = (rrow0 + 4 * i < p.M) ? *reinterpret_cast<const float4*>(p.resid + (long)(rrow0 + 4 * i) * p.ldc + rcol)
-                                                          : make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
                     uint32_t ra[32];
                     float v[32];
                     umma::tmem_ld32(taddr + c0, ra);
@@ -828,6 +835,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                             *cell = o;
                         }
                     }
+                    if (c0 + 32 < (half + 1) * (BN / 2)) load_rs(c0 + 32);   // the next group's residual, in flight from here on
                     umma::fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0 && col < p.N && m * BM + q * 32 < p.M) {
