@@ -49,6 +49,7 @@ typedef enum {
 #define SVDMLP_FLAG_DECODE_COOPERATIVE 0x400u /* small T: cooperative launch of the persistent kernel (residency guaranteed by the driver) instead of a programmatic dependent launch */
 #define SVDMLP_FLAG_TOKEN_SLABS 0x800u /* large T: gate/up and the first down product run over token slabs whose H (64 MB) stays in L2; off by default (slower as measured) */
 #define SVDMLP_FLAG_NO_FUSED_DOWN1 0x1000u /* large T, ranks <= 128: gate/up and the first down product as two kernels with H in global memory, not the one fused kernel */
+#define SVDMLP_FLAG_NO_CLUSTER_SPLITK 0x2000u /* large T: split-K sums through fp32 partials and a reduction launch, never through distributed shared memory inside a cluster */
 #define SVDMLP_FLAG_NO_WIDE_GATEUP 0x200u /* large T, ranks > 256: gate/up on 128-wide tiles, not 256-wide ones */
 
 /*

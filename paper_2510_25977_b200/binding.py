@@ -22,6 +22,7 @@ FLAG_DECODE_REGISTERS = 0x40
 FLAG_NO_CTA_PAIRS = 0x80
 FLAG_NO_TMEM_STRIP = 0x100
 FLAG_NO_WIDE_GATEUP = 0x200
+FLAG_NO_CLUSTER_SPLITK = 0x2000
 FLAG_DECODE_COOPERATIVE = 0x400
 FLAG_TOKEN_SLABS = 0x800
 FLAG_NO_FUSED_DOWN1 = 0x1000

@@ -188,7 +188,8 @@ int launch_gemm_pair_t(const GemmPlan& g, cudaStream_t s) {
     cfg.gridDim = dim3(g.grid); cfg.blockDim = dim3(tensorpath::kPairThreads); cfg.dynamicSmemBytes = g.smem; cfg.stream = s;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[0].val.clusterDim.x = 2 * std::max(1, g.p.cks);   // one CTA pair, or the pairs that split K among themselves
+    attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 2;
@@ -346,7 +347,7 @@ size_t part_elems_for(int max_T, int R, int r_gate, int r_down) {
 // Fill the shape-dependent part of a plan (tensor maps are set by the caller).
 // want_res: keep the A strip resident if it fits.  allow_split: use split-K to fill the machine.
 void plan_gemm(GemmPlan& g, int nb, int bn, bool want_res, bool allow_split, int M, int N, int K, int batch,
-               bool c_tma = false, bool want_pair = false, int force_ksplit = 0) {
+               bool c_tma = false, bool want_pair = false, int force_ksplit = 0, bool allow_cluster = false) {
     using namespace tensorpath;
     g.nb = nb; g.bn = bn; g.pair = false;
     GemmParams& p = g.p;
@@ -400,7 +401,24 @@ void plan_gemm(GemmPlan& g, int nb, int bn, bool want_res, bool allow_split, int
         g.pair = true;
     }
     p.split_stride = 0; p.batch_col_off = 0; p.resid = nullptr;
-    p.a_mn = 0; p.c_t = 0;
+    p.a_mn = 0; p.c_t = 0; p.cks = 0;
+    // Two splits on CTA pairs: the two pairs that split a tile's K range form one cluster of four CTAs and sum their
+    // accumulators through distributed shared memory; the fp32 partial buffer and the reduction launch disappear
+    // (config 3: first projection at T = 2048 16.6 -> 14.7 us, first down product at T = 8192 53.9 -> 46.2 us).
+    // One tile per cluster (the receive buffers are the ring), 16-bit output only.  Four pairs per cluster (the
+    // kernel supports it) measured twice as slow as four partials and a reduction launch (T = 4096: 47.6 against
+    // 33.1 us): clusters of eight CTAs do not all become resident at once.
+    if (allow_cluster && g.pair && !g.ares && nb == 1 && force_ksplit == 0 && p.ksplit == 2) {
+        const int cks = 2;
+        const int tiles = ((p.tiles_m + 1) / 2) * p.tiles_n * batch;
+        const size_t ring_bytes = (size_t)p.stages * (size_t)std::max(1, p.cps) * (kABytes + (size_t)bn / 2 * BK * 2);
+        const size_t recv_bytes = (size_t)BM * bn * 4;   // [split][128 rows][bn / cks floats]
+        const int cps_k = (p.chunks_total + cks - 1) / cks;
+        if (tiles * cks <= num_sms() / 2 && recv_bytes <= ring_bytes && (cks - 1) * cps_k < p.chunks_total) {
+            p.cks = cks; p.ksplit = 1; p.chunks_per_split = cps_k;
+            g.grid = 2 * cks * tiles;
+        }
+    }
     if (!(g.pair && !g.ares)) p.cps = 1;
 }
 
@@ -760,7 +778,7 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     // ranks that are whole 256-column tiles, with enough tiles to fill the machine without splitting K: 256 x 256 pair
     // tiles halve the re-reads of X (r = 256, T = 8192: 34.5 -> 29.5 us; with fewer tiles the split and its sum cost more)
     const int bn1 = (pairs_ok && h->rg >= 256 && h->rg % 256 == 0 && (long)((T + 255) / 256) * (h->rg / 256) * 2 >= 48) ? 256 : 128;
-    plan_gemm(g, 1, bn1, false, true, T, h->rg, h->d, 2, false, pairs_ok);
+    plan_gemm(g, 1, bn1, false, true, T, h->rg, h->d, 2, false, pairs_ok, 0, !(h->flags & SVDMLP_FLAG_NO_CLUSTER_SPLITK));
     g.p.tmA[0] = h->mX; g.p.tmA[1] = h->mX;
     g.p.tmB[0] = g.pair ? (bn1 == 256 ? h->mVg128 : h->mVg64) : h->mVg; g.p.tmB[1] = g.pair ? (bn1 == 256 ? h->mVu128 : h->mVu64) : h->mVu;
     g.p.a_fmt = umma::kFmtBF16; g.p.b_fmt = umma::kFmtBF16; g.p.status = h->status_dev;
@@ -788,6 +806,7 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     const SlabPlan* sp = slab_plan(h, T);
     if (sp == nullptr) return SVDMLP_ERR_CUDA;
     int down1_ksplit = 0;
+    bool down1_in_cluster = false;
     // Ranks up to 128: both products in one kernel, H stays in shared memory (mlp_fused_ts.cuh)
     const int fused_S = ((mask & 6u) == 6u && sp->n == 1) ? fused_plan(h, T) : 0;
     if (fused_S > 0) {
@@ -839,20 +858,27 @@ int tensor_forward(svdmlp* h, const __nv_bfloat16* X, int T, void* Y, int y_fp32
     }
     if (mask & 4u) {
     const int bn3 = down1_tile_width(h->rd);
-    plan_gemm(g, 1, bn3, false, true, Ts, h->rd, h->ffn, 1, false, pairs_ok, down1_ksplit);
+    // (the sum inside a cluster writes fp16 Zd itself: not when the caller wants the fp32 sum, not with token slabs)
+    const bool cl_ok = sp->n == 1 && h->zd_out32 == nullptr && !(h->flags & SVDMLP_FLAG_NO_CLUSTER_SPLITK);
+    plan_gemm(g, 1, bn3, false, true, Ts, h->rd, h->ffn, 1, false, pairs_ok, down1_ksplit, cl_ok);
     if (si == 0) down1_ksplit = g.p.ksplit;
     if (g.p.ksplit != down1_ksplit) return SVDMLP_ERR_UNSUPPORTED;  // cannot happen: the split depends on K alone once forced
     g.p.tmA[0] = sm.h; g.p.tmA[1] = sm.h;
     g.p.tmB[0] = g.pair ? h->mVdHalf : h->mVd; g.p.tmB[1] = g.p.tmB[0];
     g.p.a_fmt = umma::kFmtF16; g.p.b_fmt = umma::kFmtF16; g.p.status = h->status_dev;
-    if ((size_t)g.p.ksplit * T * h->rd > h->part_elems) return SVDMLP_ERR_NOMEM;
-    g.p.C = h->part + (size_t)row0 * h->rd; g.p.ldc = h->rd; g.p.split_stride = (long)T * h->rd; g.p.out_mode = OUT_F32;
+    down1_in_cluster = g.p.cks > 1;
+    if (down1_in_cluster) {
+        g.p.C = h->Zd16; g.p.ldc = h->rd; g.p.out_mode = OUT_F16;
+    } else {
+        if ((size_t)g.p.ksplit * T * h->rd > h->part_elems) return SVDMLP_ERR_NOMEM;
+        g.p.C = h->part + (size_t)row0 * h->rd; g.p.ldc = h->rd; g.p.split_stride = (long)T * h->rd; g.p.out_mode = OUT_F32;
+    }
     { ProfScope ps(h, "down1", s); rc = launch_gemm(g, s); }
     if (rc != SVDMLP_OK) return rc;
     h->launches += 1;
     }
     }
-    if (mask & 4u) {
+    if ((mask & 4u) && !down1_in_cluster) {
     { ProfScope ps(h, "down1_reduce", s); rc = launch_reduce(h->part, down1_ksplit, (long)T * h->rd, (long)T * h->rd, h->Zd16, s, h->zd_out32); }
     if (rc != SVDMLP_OK) return rc;
     h->launches += 1;

@@ -52,6 +52,10 @@ struct GemmParams {
     // Layout flags of the XUV operator (Algorithm 2's is_XT / req_OT); streaming one-branch kernels only.
     int a_mn;            // 1: A is given transposed, A^T[K, M]: tmA has boxes [64 k][64 m], the tile is an MN-major operand
     int c_t;             // 1: the 16-bit TMA-store epilogue writes C^T[N, M]: tmC has boxes [64 n][32 m], no swizzle
+    // Split-K inside a cluster (streaming one-branch CTA-pair kernel only): the cluster is cks CTA pairs, pair s takes
+    // K split s of the cluster's one tile, and the partial accumulators are summed through distributed shared memory
+    // (no partial buffer, no reduction launch).  0 or 1: off.
+    int cks;
 };
 
 __device__ __forceinline__ float fast_silu(float g) {
@@ -555,18 +559,25 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = umma::cluster_ctarank();
+    // Cluster = one CTA pair, or (split-K inside the cluster) cks pairs that share a tile: crank = 2 split + rank.
+    const uint32_t crank = umma::cluster_ctarank();
+    const int cks = (!ARES && NB == 1 && p.cks > 1) ? p.cks : 1;
+    const uint32_t rank = crank & 1u;        // rank within the pair
+    const uint32_t lead = crank & ~1u;       // cluster rank of the pair's leader
+    const int split = (int)(crank >> 1);
+    const uint16_t pair_mask = (uint16_t)(3u << lead);
     const bool leader = rank == 0;
-    const int cluster_id = blockIdx.x >> 1, nclusters = gridDim.x >> 1;
+    const int cluster_id = blockIdx.x / (2 * cks), nclusters = gridDim.x / (2 * cks);
     const int pairs_m = (p.tiles_m + 1) / 2;
-    const int total_tiles = pairs_m * p.tiles_n * p.batch * p.ksplit;
-    const int per_cluster = (total_tiles + nclusters - 1) / nclusters;
+    const int total_tiles = pairs_m * p.tiles_n * p.batch * p.ksplit;   // ksplit = 1 with split-K inside the cluster
+    const int per_cluster = (total_tiles + nclusters - 1) / nclusters;  // 1 with split-K inside the cluster
     const int tile_begin = cluster_id * per_cluster;
     const int tile_end = min(total_tiles, tile_begin + per_cluster);
     // tile index -> (row-strip pair, column tile, split-K part, batch entry)
     auto decode = [&](int t, int& mp, int& n, int& ks, int& z) {
         if (ARES) { mp = t / p.tiles_n; n = t - mp * p.tiles_n; ks = 0; z = 0; }
         else { n = t % p.tiles_n; t /= p.tiles_n; mp = t % pairs_m; t /= pairs_m; ks = t % p.ksplit; z = t / p.ksplit; }
+        if (cks > 1) ks = split;   // chunks_per_split is the cluster's split size
     };
 
     if (threadIdx.x == 0) {
@@ -598,6 +609,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                 umma::tma_prefetch_2d(&p.tmB[NB == 2 ? b : z], c * BK, n * BN + (int)rank * (BN / 2));
     }
     umma::pdl_wait();
+    bool cl_ready = false;   // split-K inside the cluster: this epilogue warp's accumulator is complete
 
     if (warp == 0 || warp == kPairProducer2) {
         // ---------------- TMA producers (both CTAs): own A strip, own half of every B chunk ----------------
@@ -616,7 +628,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                 if (cur_mp >= 0) { ok = umma::mbar_wait_warp(aempty, a_phase, abort_flag); a_phase ^= 1; if (!ok) break; }
                 if (umma::elect_one()) {
                     if (leader) umma::mbar_expect_tx(afull, 2 * NB * a_chunks * kABytes);
-                    const uint32_t bar = umma::map_to_rank(afull, 0);
+                    const uint32_t bar = umma::map_to_rank(afull, lead);
                     for (int b = 0; b < NB; ++b)
                         for (int c = 0; c < a_chunks; ++c)
                             umma::tma_load_2d_pair(a_res + (b * a_chunks + c) * kABytes, &p.tmA[b], bar, c * BK, m * BM);
@@ -635,7 +647,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                     if (!ok) break;
                     if (umma::elect_one()) {
                         if (leader) umma::mbar_expect_tx(&full[stage], 2 * slot_bytes);
-                        const uint32_t bar = umma::map_to_rank(&full[stage], 0);
+                        const uint32_t bar = umma::map_to_rank(&full[stage], lead);
                         unsigned char* st = ring + stage * slot_bytes;
                         if (ARES) {
 #pragma unroll
@@ -715,7 +727,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                                         umma::mma_f16_ss_pair(dcol, ad + a_step * kk, bd + 2 * kk, idesc,
                                                               (c + j > c_begin) || (kk > 0));
                                 }
-                            umma::mma_commit_pair(&empty[stage]);
+                            umma::mma_commit_pair(&empty[stage], pair_mask);
                         }
                         __syncwarp();
                         if (++stage == p.stages) { stage = 0; phase ^= 1; }
@@ -724,8 +736,8 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
                 if (!ok) break;
                 const bool last_of_m = ARES && ((t + 1 == tile_end) || (n + 1 == p.tiles_n));
                 if (umma::elect_one()) {
-                    umma::mma_commit_pair(&tfull[acc]);
-                    if (last_of_m) umma::mma_commit_pair(aempty);
+                    umma::mma_commit_pair(&tfull[acc], pair_mask);
+                    if (last_of_m) umma::mma_commit_pair(aempty, pair_mask);
                 }
                 __syncwarp();
                 if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
@@ -745,7 +757,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
         const int esz = (p.out_mode == OUT_F32) ? 4 : 2;
         const bool f16_out = p.out_mode == OUT_F16;
         unsigned char* my_stage = stage_out + (warp - 2) * 4096;
-        const uint32_t tempty_leader[2] = {umma::map_to_rank(&tempty[0], 0), umma::map_to_rank(&tempty[1], 0)};
+        const uint32_t tempty_leader[2] = {umma::map_to_rank(&tempty[0], lead), umma::map_to_rank(&tempty[1], lead)};
         // The residual rows this warp will add are requested into L2 one tile ahead (the first tile's at kernel
         // start): read on demand, each 32-column group waited a full HBM round trip inside the epilogue.
         auto prefetch_resid = [&](int tt) {
@@ -780,6 +792,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
             ok = umma::mbar_wait_warp(&tfull[acc], acc ? acc_phase1 : acc_phase0, abort_flag);
             if (!ok) break;
             umma::tc_fence_after_sync();
+            if (cks > 1) { cl_ready = true; break; }   // the sum over the cluster's splits follows below, for all roles together
             const int row = m * BM + q * 32 + lane;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * ACC_COLS;
             // The accumulator goes back to the issuer as soon as this warp's last TMEM load has landed in
@@ -942,6 +955,65 @@ __global__ void __launch_bounds__(kPairThreads, 1) gemm_pair_kernel(const __grid
         if (p.c_tma) umma::bulk_wait_all();
     }
 
+    if (cks > 1) {
+        // ---- split-K inside the cluster: reduce-scatter of the cks partial accumulators through distributed shared memory.
+        // Pair s owns the columns [s W, (s + 1) W) of the tile, W = BN / cks.  Every epilogue thread pushes its row's 32-column
+        // groups into the owner's receive buffer (the ring, idle by now): [source split][128 rows][W floats + 4 of padding];
+        // then every CTA sums its W columns over the sources in split order (a fixed order: the result does not depend on
+        // timing) and stores them.  Both cluster barriers are reached by every thread of every CTA, whatever happened before.
+        // Receive layout: [source split][32-row block][16-byte piece of the W columns][row in block][4 floats], so that a
+        // warp instruction (lane = row) writes, and later reads, 512 contiguous bytes.
+        const int W = BN / cks, blk = W * 128;        // bytes of one 32-row block: W / 4 pieces x 512 B
+        umma::cluster_sync();   // every CTA's MMAs have finished reading its ring
+        const bool epi = warp >= 2 && warp < 2 + kEpiWarps;
+        if (epi && cl_ready) {
+            const int q = warp & 3, half = (warp - 2) >> 2;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+                uint32_t ra[32];
+                umma::tmem_ld32(taddr + c0, ra);
+                umma::tmem_ld_wait();
+                const int owner = c0 / W, cw = c0 - owner * W;   // a 32-column group never straddles two owners (W >= 32)
+                const uint32_t dst = umma::map_to_rank(ring + (size_t)(split * 4 + q) * blk + (cw / 4) * 512 + lane * 16, 2u * owner + rank);
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    umma::st_cluster_f32x4(dst + 512 * j, __uint_as_float(ra[4 * j]), __uint_as_float(ra[4 * j + 1]),
+                                           __uint_as_float(ra[4 * j + 2]), __uint_as_float(ra[4 * j + 3]));
+            }
+        }
+        umma::cluster_sync();   // all pushes have landed (release / acquire at cluster scope)
+        if (epi && tile_begin < tile_end) {
+            int mp, n, ks, z;
+            decode(tile_begin, mp, n, ks, z);
+            const int te = threadIdx.x - 64, r = te & (BM - 1), part = te >> 7;   // 256 threads: row, column half of the slice
+            const int row = (2 * mp + (int)rank) * BM + r, hw = W / 2;
+            const int col0 = n * BN + split * W + part * hw;
+            if (row < p.M) {
+                char* out = reinterpret_cast<char*>(p.C) + ((long)row * p.ldc + (long)z * p.batch_col_off + col0) * 2;
+                for (int c = 0; c < hw; c += 8) {
+                    float acc8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    for (int src = 0; src < cks; ++src) {
+                        const unsigned char* cell = ring + (size_t)(src * 4 + (r >> 5)) * blk + ((part * hw + c) / 4) * 512 + (r & 31) * 16;
+                        const float4 a = *reinterpret_cast<const float4*>(cell), b = *reinterpret_cast<const float4*>(cell + 512);
+                        acc8[0] += a.x; acc8[1] += a.y; acc8[2] += a.z; acc8[3] += a.w;
+                        acc8[4] += b.x; acc8[5] += b.y; acc8[6] += b.z; acc8[7] += b.w;
+                    }
+                    if (col0 + c + 8 <= p.N) {
+                        uint4 w;
+                        if (p.out_mode == OUT_F16) {
+                            w.x = pack_f16(acc8[0], acc8[1]); w.y = pack_f16(acc8[2], acc8[3]);
+                            w.z = pack_f16(acc8[4], acc8[5]); w.w = pack_f16(acc8[6], acc8[7]);
+                        } else {
+                            w.x = pack_bf16(acc8[0], acc8[1]); w.y = pack_bf16(acc8[2], acc8[3]);
+                            w.z = pack_bf16(acc8[4], acc8[5]); w.w = pack_bf16(acc8[6], acc8[7]);
+                        }
+                        *reinterpret_cast<uint4*>(out + c * 2) = w;
+                    }
+                }
+            }
+        }
+    }
     umma::tc_fence_before_sync();
     __syncthreads();
     if (*abort_flag) {

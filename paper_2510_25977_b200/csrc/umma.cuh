@@ -222,10 +222,13 @@ __device__ __forceinline__ void mma_f16_ss_pair(uint32_t d_tmem, uint64_t adesc,
 }
 // Arrive on the barrier at this shared-memory offset in both CTAs of the pair once all MMAs issued
 // so far have completed.
-__device__ __forceinline__ void mma_commit_pair(uint64_t* bar) {
-    const uint16_t mask = 3;
+__device__ __forceinline__ void mma_commit_pair(uint64_t* bar, uint16_t mask = 3) {   // mask: cluster ranks of the two CTAs
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                  ::"r"(smem_u32(bar)), "h"(mask) : "memory");
+}
+// 16-byte store into the shared memory of another CTA of the cluster (address from map_to_rank)
+__device__ __forceinline__ void st_cluster_f32x4(uint32_t cluster_addr, float a, float b, float c, float d) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
 // ---- descriptors ----------------------------------------------------------------------------

@@ -143,6 +143,21 @@ def test_between_9_and_32_tokens_the_path_follows_the_decode_kernels_fit(oracle,
     _gpu.assert_close(Y, _gpu.oracle_rows(oracle, f, X, list(range(T))), f"T={T} r={r} ({path})")
 
 
+@pytest.mark.parametrize("T", [2048, 1900])
+def test_split_k_summed_inside_a_cluster(oracle, T):
+    """Two K splits of the first projection on CTA pairs form one cluster and are summed through distributed shared
+    memory (d = 1024 is 16 K chunks: exactly two splits at these T).  Against the oracle, every row, and against the
+    same handle shape with the partial-buffer + reduction-launch form: both sum split 0 then split 1 in fp32, so the
+    two forms give the same bits."""
+    d, ffn, r = 1024, 2048, 256
+    f = inputs.direct_factors(d, ffn, r, seed=8, device="cuda")
+    X = inputs.activations(T, d, seed=8, device="cuda")
+    Y = _gpu.run_mlp(f, X)
+    Y_plain = _gpu.run_mlp(f, X, flags=binding.FLAG_NO_CLUSTER_SPLITK)
+    _gpu.assert_close(Y, _gpu.oracle_rows(oracle, f, X, list(range(T))), f"cluster split-K T={T}")
+    assert torch.equal(Y, Y_plain)
+
+
 @pytest.mark.parametrize("T", [1, 8, 1024])
 def test_cfg5_prenorm_residual_stack(oracle, T):
     d, ffn, r, L = 5120, 13824, 320, 40
