@@ -344,6 +344,25 @@ size_t part_elems_for(int max_T, int R, int r_gate, int r_down) {
     return n;
 }
 
+// How many clusters of four CTAs (two CTA pairs) of the streaming pair kernel can be resident at once: fewer than
+// SMs / 4, because a cluster must fit inside one GPC (B200: 33 of 37; clusters of eight: 15 of 18).
+int max_active_clusters4() {
+    static int n = -1;
+    if (n < 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(4 * 64); cfg.blockDim = dim3(tensorpath::kPairThreads); cfg.dynamicSmemBytes = kSmemBudget + 1024;
+        cudaLaunchAttribute a[1];
+        a[0].id = cudaLaunchAttributeClusterDimension;
+        a[0].val.clusterDim.x = 4; a[0].val.clusterDim.y = 1; a[0].val.clusterDim.z = 1;
+        cfg.attrs = a; cfg.numAttrs = 1;
+        int v = 0;
+        cudaFuncSetAttribute(tensorpath::gemm_pair_kernel<1, 256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024);
+        if (cudaOccupancyMaxActiveClusters(&v, tensorpath::gemm_pair_kernel<1, 256, false>, &cfg) != cudaSuccess) { cudaGetLastError(); v = 0; }
+        n = v;
+    }
+    return n;
+}
+
 // Fill the shape-dependent part of a plan (tensor maps are set by the caller).
 // want_res: keep the A strip resident if it fits.  allow_split: use split-K to fill the machine.
 void plan_gemm(GemmPlan& g, int nb, int bn, bool want_res, bool allow_split, int M, int N, int K, int batch,
@@ -407,14 +426,15 @@ void plan_gemm(GemmPlan& g, int nb, int bn, bool want_res, bool allow_split, int
     // (config 3: first projection at T = 2048 16.6 -> 14.7 us, first down product at T = 8192 53.9 -> 46.2 us).
     // One tile per cluster (the receive buffers are the ring), 16-bit output only.  Four pairs per cluster (the
     // kernel supports it) measured twice as slow as four partials and a reduction launch (T = 4096: 47.6 against
-    // 33.1 us): clusters of eight CTAs do not all become resident at once.
+    // 33.1 us): at most 15 clusters of eight CTAs are resident at once (a cluster must fit inside a GPC) and every
+    // shape here has 16 tiles; clusters of four: 33.
     if (allow_cluster && g.pair && !g.ares && nb == 1 && force_ksplit == 0 && p.ksplit == 2) {
         const int cks = 2;
         const int tiles = ((p.tiles_m + 1) / 2) * p.tiles_n * batch;
         const size_t ring_bytes = (size_t)p.stages * (size_t)std::max(1, p.cps) * (kABytes + (size_t)bn / 2 * BK * 2);
         const size_t recv_bytes = (size_t)BM * bn * 4;   // [split][128 rows][bn / cks floats]
         const int cps_k = (p.chunks_total + cks - 1) / cks;
-        if (tiles * cks <= num_sms() / 2 && recv_bytes <= ring_bytes && (cks - 1) * cps_k < p.chunks_total) {
+        if (tiles <= max_active_clusters4() && recv_bytes <= ring_bytes && (cks - 1) * cps_k < p.chunks_total) {
             p.cks = cks; p.ksplit = 1; p.chunks_per_split = cps_k;
             g.grid = 2 * cks * tiles;
         }
