@@ -1,8 +1,8 @@
 // Exchange step of the tensor-parallel forward (Section 4.2.2, Figure 4: the one all-reduce of the partitioned MLP;
 // with factored weights it falls on the narrow fp32 Zd[T, r_down]).  No collective library: every rank PUSHES its
 // partial into its slot of every peer's receive buffer with plain peer stores and then raises a flag per peer;
-// the consumer waits (bounded) for the G flags of the step and sums the G slots.  Nothing here is a multicast or a
-// bulk copy; the peers' buffers are ordinary peer-mapped device memory.
+// the consumer waits (bounded) for the G flags of the step and sums the G slots.  The only accesses to a
+// peer's memory are ordinary st.global / ld.global on peer-mapped device memory.
 //
 // Receive buffer of a rank: float [2][G][slot] (slot = max_T * r_down), the first index = step parity.  Two
 // buffers are enough: a peer pushes step e + 2 only after it has gathered step e + 1, which needed this rank's push

@@ -1,5 +1,5 @@
-// Thin wrappers over the sm_100a PTX this library is built on: mbarrier, TMA tiled copies
-// (cp.async.bulk.tensor, never with cluster multicast), tcgen05 MMA / TMEM management, and the
+// Thin wrappers over the sm_100a PTX this library is built on: mbarrier, TMA tiled copies (every load is
+// addressed to one CTA's shared memory), tcgen05 MMA / TMEM management, and the
 // descriptor encodings they consume.  Every wait is bounded: it gives up after a wall-clock
 // limit, raises the CTA's abort flag and lets the kernel tear down normally.
 #pragma once
